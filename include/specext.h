@@ -1,0 +1,155 @@
+/*
+ * specext.h -- C ABI of the verification hot path of speculative decoding with Cross-model
+ * Retrieval: Hybrid Tree Attention fused with the per-chunk attention mass that retrieval ranks,
+ * top-k chunk selection, and the gather that rewrites the draft model's KV cache.
+ *
+ * General conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library never allocates,
+ *     frees or synchronises on these calls; all work is enqueued on `cuda_stream` (a cudaStream_t
+ *     passed as void*, NULL = the legacy default stream) and the call returns at once.
+ *   - The return value is the result of synchronous host-side argument checking (a
+ *     specext_status).  Problems only the device can see (an invalid parent[] entry, a bounded
+ *     wait that ran out) are OR-ed as (1 << status) into *device_status, an int32 in device
+ *     memory that the caller zeroes once and may read after synchronising; outputs are then
+ *     unspecified, but every kernel terminates.
+ *   - bf16 tensors are raw 16-bit patterns.  The innermost dimension (head_dim) is contiguous;
+ *     all other strides are given in elements, must be multiples of 8 elements (16 bytes), and
+ *     base pointers must be 16-byte aligned.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - Calls that share a workspace or outputs must be ordered by the stream.
+ */
+#ifndef SPECEXT_H_
+#define SPECEXT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPECEXT_OK = 0,
+  SPECEXT_ERR_INVALID_ARG = 1, /* null / misaligned pointer, size or stride out of range        */
+  SPECEXT_ERR_UNSUPPORTED = 2, /* shape outside what the kernels are built for                   */
+  SPECEXT_ERR_WORKSPACE = 3,   /* workspace_bytes smaller than specext_verify_attn_workspace()   */
+  SPECEXT_ERR_BAD_TREE = 4,    /* device: parent[i] outside [-1, i-1]                            */
+  SPECEXT_ERR_TIMEOUT = 5,     /* device: a bounded wait inside a kernel expired                 */
+  SPECEXT_ERR_CUDA = 6         /* a CUDA runtime / driver call failed (launch, tensor map, ...)  */
+} specext_status;
+
+/* Shape of one verification attention call (one layer, one sequence). */
+typedef struct {
+  int32_t n_q_heads;       /* Hq                                                              */
+  int32_t n_kv_heads;      /* Hkv; Hq % Hkv == 0 and G = Hq/Hkv a power of two <= 64          */
+  int32_t head_dim;        /* D: 64 or 128                                                    */
+  int32_t prefix_len;      /* L >= 0: number of valid tokens in the prefix KV cache           */
+  int32_t n_tree;          /* T: draft-tree nodes, 1..64                                      */
+  int32_t chunk_size;      /* C: tokens per retrieval chunk, a power of two in 1..128         */
+  float softmax_scale;     /* multiplies q.k before the softmax; 0 selects 1/sqrt(D)          */
+  int32_t want_chunk_score;/* non-zero: also produce chunk_score (the last layer only)        */
+  int64_t q_stride_t, q_stride_h;     /* Q      [T][Hq][D]                                    */
+  int64_t kv_stride_l, kv_stride_h;   /* K_prefix and V_prefix [>=L][Hkv][D], same strides    */
+  int64_t tkv_stride_t, tkv_stride_h; /* K_tree and V_tree [T][Hkv][D], same strides          */
+  int64_t o_stride_t, o_stride_h;     /* O      [T][Hq][D]                                    */
+} specext_attn_desc;
+
+/*
+ * Bytes of scratch that specext_verify_attn needs for this shape (0 on an invalid descriptor).
+ * The scratch holds the per-split partial results of the split-over-KV attention and is fully
+ * rewritten by every call; 256-byte alignment is required.
+ */
+size_t specext_verify_attn_workspace(const specext_attn_desc* desc);
+
+/*
+ * Hybrid Tree Attention of the target model's verification step (Section 3.1, "Efficient
+ * Attention") together with the attention scores that Cross-model Retrieval ranks chunks by
+ * (Section 3.2.1, "Method Overview"; the scores of the last layer of the most recent
+ * verification pass).
+ *
+ * For every tree node t and query head h, with g = h / G:
+ *   s_j = scale * <Q[t,h], K_prefix[j,g]>            for the L prefix tokens,
+ *   s_u = scale * <Q[t,h], K_tree[u,g]>              for tree nodes u that are t itself or an
+ *                                                    ancestor of t (others are masked out),
+ *   P = softmax over all visible keys, O[t,h] = sum P * V, lse[h,t] = log sum exp(s),
+ *   chunk_score[t,c] = (1/Hq) * sum_h sum_{j in chunk c} P_j,  chunk c = tokens [cC, min(L,(c+1)C)).
+ * The prefix is processed in splits along the KV length with an online softmax and the partial
+ * results are merged by log-sum-exp, so the result equals unsplit attention up to rounding.
+ *
+ *   Q, K_prefix, V_prefix, K_tree, V_tree : bf16, layouts as in the descriptor.  Memory of the
+ *       prefix cache beyond prefix_len is never read.
+ *   parent      : int32 [T]; parent[i] is the tree index of node i's parent, -1 when the parent is
+ *                 the last prefix token.  Must satisfy -1 <= parent[i] < i (else BAD_TREE).
+ *   O           : bf16 [T][Hq][D] (strides from the descriptor), rounded once from fp32.
+ *   lse         : fp32 [Hq][T], natural logarithm, softmax_scale included.
+ *   chunk_score : fp32 [T][ceil(L/C)], written only when want_chunk_score != 0 (may be NULL
+ *                 otherwise).
+ *   workspace   : scratch of at least specext_verify_attn_workspace(desc) bytes.
+ * Arithmetic: bf16 products accumulated in fp32; probabilities are rounded to bf16 for the
+ * P*V product; chunk sums and the normaliser are accumulated in fp32 from unrounded exponentials.
+ */
+int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void* K_prefix,
+                        const void* V_prefix, const void* K_tree, const void* V_tree,
+                        const int32_t* parent, void* O, float* lse, float* chunk_score,
+                        void* workspace, size_t workspace_bytes, int32_t* device_status,
+                        void* cuda_stream);
+
+/*
+ * SelectChunks of Algorithm 1 (Appendix A; Section 3.2.1: rank the fixed-size chunks of the
+ * prefix by their average attention score for one query and keep the top k).
+ *
+ *   chunk_score : fp32 [n_tree][n_chunks] as written by specext_verify_attn.
+ *   row         : which tree node's scores to rank (the last accepted token), 0 <= row < n_tree.
+ *   prefix_len, chunk_size : define n_chunks = ceil(L/C) (must equal the argument) and the
+ *                 length len_c of the trailing chunk.  Any chunk_size >= 1 is accepted.
+ *   k           : number of chunks to keep, >= 1; k_eff = min(k, n_chunks).
+ *   idx         : int32 [min(k, n_chunks)] out, the kept chunk indices in ascending order.
+ *   n_selected  : int32 [1] out (device), = k_eff.
+ * Ranking key: chunk_score[row][c] / (float)len_c in fp32 (IEEE division); larger first, equal
+ * keys ordered by lower chunk index.  Scores must be finite and non-negative.
+ * n_chunks <= 65536.
+ */
+int specext_select_chunks(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t* idx,
+                          int32_t* n_selected, int32_t* device_status, void* cuda_stream);
+
+/*
+ * UpdateDraftCache of Algorithm 1 (Appendix A; Section 3.2.1: the draft model keeps only the
+ * selected chunks in its KV cache).  Copies the selected chunks of the draft model's K and V,
+ * bit for bit and in the order of idx, into a compact cache.
+ *
+ *   draft_K, draft_V : bf16 [n_layers][>=L][n_kv_heads][head_dim] with element strides
+ *                      stride_layer, stride_l, stride_h (head_dim contiguous).
+ *   idx, n_selected  : device outputs of specext_select_chunks (ascending chunk indices, each in
+ *                      [0, ceil(L/C)) -- entries outside that range are skipped and reported as
+ *                      INVALID_ARG in *device_status).
+ *   max_selected     : upper bound on *n_selected that sizes the launch (the k passed to select).
+ *   K_out, V_out     : bf16 [n_layers][max_selected*C][n_kv_heads][head_dim], contiguous; token
+ *                      slot i*C + o receives token idx[i]*C + o.  Only a trailing chunk can be
+ *                      short, and it can only come last, so the valid tokens are contiguous.
+ *   n_tokens_out     : int32 [1] out (device): number of valid tokens written per layer.
+ * n_kv_heads * head_dim must be a multiple of 8 (16-byte vectors).
+ */
+int specext_gather_kv(const void* draft_K, const void* draft_V, int32_t n_layers,
+                      int32_t n_kv_heads, int32_t head_dim, int32_t prefix_len, int32_t chunk_size,
+                      int64_t stride_layer, int64_t stride_l, int64_t stride_h, const int32_t* idx,
+                      const int32_t* n_selected, int32_t max_selected, void* K_out, void* V_out,
+                      int32_t* n_tokens_out, int32_t* device_status, void* cuda_stream);
+
+/*
+ * Copies *device_status to the host after synchronising the stream and returns it (a bit set of
+ * 1 << specext_status), or -SPECEXT_ERR_CUDA if the copy failed.  For tests and debugging; not
+ * part of the asynchronous path.
+ */
+int specext_read_status(const int32_t* device_status, void* cuda_stream);
+
+/* Static, human-readable name of a specext_status value. */
+const char* specext_status_string(int status);
+
+/* Number of kernels the library has launched in this process (all calls, all streams). */
+int64_t specext_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECEXT_H_ */

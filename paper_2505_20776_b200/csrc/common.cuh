@@ -1,0 +1,60 @@
+// Shared device/host declarations of the specext kernels.
+#ifndef SPECEXT_COMMON_CUH_
+#define SPECEXT_COMMON_CUH_
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/specext.h"
+#include "plan.h"
+
+struct AttnArgs {
+  AttnPlan plan;
+  const __nv_bfloat16* Q;
+  const __nv_bfloat16* Kp;
+  const __nv_bfloat16* Vp;
+  const __nv_bfloat16* Kt;
+  const __nv_bfloat16* Vt;
+  const int32_t* parent;
+  __nv_bfloat16* O;
+  float* lse;
+  float* chunk_score;
+  float* ws;
+  int32_t* status;
+  long long q_st, q_sh, kv_sl, kv_sh, tkv_st, tkv_sh, o_st, o_sh;
+};
+
+__device__ __forceinline__ void spx_raise(int32_t* status, int code) {
+  if (status) atomicOr(status, 1 << code);
+}
+
+// Ancestor-or-self bit masks of the draft tree: bit u of anc[t] is set iff u == t or u is a
+// proper ancestor of t.  Each of the first T threads walks up from its own node; a parent outside
+// [-1, t-1] raises BAD_TREE and ends the walk, so the loop is bounded by T steps.
+__device__ __forceinline__ void spx_build_ancestors(const int32_t* __restrict__ parent, int T,
+                                                    unsigned long long* anc_smem, int32_t* status) {
+  const int t = threadIdx.x;
+  if (t < 64) {
+    unsigned long long m = 0;
+    if (t < T) {
+      int u = t;
+      for (int step = 0; step <= T && u >= 0; ++step) {
+        m |= 1ull << u;
+        const int p = parent[u];
+        if (p < -1 || p >= u) {
+          spx_raise(status, SPECEXT_ERR_BAD_TREE);
+          break;
+        }
+        u = p;
+      }
+    }
+    anc_smem[t] = m;
+  }
+}
+
+// Launchers implemented in the kernel translation units; each returns the cudaError_t of its launch.
+cudaError_t spx_launch_attn_simt(const AttnArgs& a, cudaStream_t st, int* n_launches);
+cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches);
+
+#endif  // SPECEXT_COMMON_CUH_

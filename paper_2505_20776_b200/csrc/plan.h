@@ -1,0 +1,56 @@
+// Work decomposition of one verification-attention call, shared by host and device code.
+//
+// Rows.  For KV head g the G = Hq/Hkv query heads that read it are stacked with the T tree
+// nodes into G*T query rows, row r = t*G + i  <->  (node t, head g*G + i).  Rows are cut into
+// row blocks of RB (128 or 256) rows; a (KV head, row block) pair is a "problem".
+//
+// Units.  The prefix is cut into key tiles of 128 tokens; the tree keys form one more tile.  A
+// problem therefore has UPP = ceil(L/128) + 1 units, the last one being the tree tile.  All
+// units of all problems are laid out in one line (problem-major) and cut into n_cta contiguous
+// ranges of nearly equal length; CTA c owns units [unit_start(c), unit_start(c+1)).  The part of
+// a CTA's range that lies inside one problem is a "segment" and yields one partial result
+// (unnormalised output, running maximum, row sum) in slot c + problem.  Slots are unique because
+// both c and the problem index are non-decreasing along the line.
+#ifndef SPECEXT_PLAN_H_
+#define SPECEXT_PLAN_H_
+
+#include <stdint.h>
+
+#if defined(__CUDACC__)
+#define SPX_HD __host__ __device__ __forceinline__
+#else
+#define SPX_HD inline
+#endif
+
+#define SPX_TILE_KEYS 128
+
+struct AttnPlan {
+  int Hq, Hkv, G, D, L, T, C;
+  int rows;        // G*T query rows per KV head
+  int RB;          // rows per row block (128 or 256)
+  int n_rblk;      // row blocks per KV head
+  int NP;          // problems = Hkv * n_rblk
+  int TPH;         // prefix key tiles per problem = ceil(L/128)
+  int UPP;         // units per problem = TPH + 1 (tree tile last)
+  int U;           // total units
+  int n_cta;       // CTAs of the attention kernel (<= U)
+  int q, rem;      // U = q*n_cta + rem
+  int n_slots;     // n_cta + NP - 1 partial slots
+  int max_segs;    // upper bound on segments per problem
+  int CPT;         // chunks per key tile = 128 / C
+  int NC;          // ceil(L/C)
+  int want_score;
+  float scale2;    // softmax_scale * log2(e)
+  // workspace offsets in floats
+  long long off_part_o, off_part_m, off_part_l, off_mass, off_mref, total_floats;
+};
+
+SPX_HD int spx_unit_start(const AttnPlan& p, int c) { return c * p.q + (c < p.rem ? c : p.rem); }
+
+// CTA that owns unit u.
+SPX_HD int spx_unit_owner(const AttnPlan& p, int u) {
+  const int big = p.rem * (p.q + 1);
+  return u < big ? u / (p.q + 1) : p.rem + (u - big) / p.q;
+}
+
+#endif  // SPECEXT_PLAN_H_

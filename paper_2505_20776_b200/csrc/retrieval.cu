@@ -1,0 +1,195 @@
+// SelectChunks and UpdateDraftCache kernels.
+//
+// select_kernel (one CTA): the ranking key of chunk c is score[c] / len_c, a non-negative fp32
+// whose bit pattern orders like the value.  A most-significant-digit radix select (4 passes of
+// 8 bits, warp-aggregated shared-memory histograms) finds the k-th largest key exactly; every
+// chunk with a larger key is kept, and of the chunks equal to it the lowest-indexed are kept
+// until k are chosen.  A block-wide ballot/popcount scan in index order then emits the kept
+// chunks in ascending order, which also implements the tie rule.
+//
+// gather_kernel: 16-byte vector copy of the kept chunks of the draft K and V into the compact cache.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+
+__device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, int c, int NC, int L, int C) {
+  const int len = (c == NC - 1) ? (L - c * C) : C;
+  float x = score[c] / (float)len;
+  if (!(x > 0.f)) x = 0.f;                 // -0, negative or NaN rank lowest
+  return __float_as_uint(x);
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ score, int NC, int L,
+                                                             int C, int k, int32_t* __restrict__ idx,
+                                                             int32_t* __restrict__ n_selected) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t s_prefix, s_need;
+  __shared__ uint32_t warp_tot[2][kSelThreads / 32];
+  __shared__ uint32_t carry[2];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int keff = min(k, NC);
+
+  // ---- radix select of the keff-th largest key --------------------------------------------
+  uint32_t prefix = 0, need = keff;        // `need` keys still to take among those matching prefix
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int c = tid; c < NC; c += kSelThreads) {
+      const uint32_t key = chunk_key(score, c, NC, L, C);
+      if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // bins from high to low: lane owns bins 255-8*lane .. 248-8*lane
+      uint32_t local[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        local[i] = hist[255 - (lane * 8 + i)];
+        tot += local[i];
+      }
+      uint32_t incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      uint32_t before = incl - tot;       // keys in strictly higher bins than this lane's
+      if (before < need && need <= incl) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (before < need && need <= before + local[i]) {
+            s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + i)) << shift);
+            s_need = need - before;
+          }
+          before += local[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = s_prefix;
+    need = s_need;
+    __syncthreads();
+  }
+  const uint32_t theta = prefix;           // the keff-th largest key
+  const uint32_t need_eq = need;           // how many keys equal to theta are kept (lowest indices)
+
+  // ---- emit in ascending index order --------------------------------------------------------
+  if (tid == 0) carry[0] = carry[1] = 0;
+  __syncthreads();
+  for (int base = 0; base < NC; base += kSelThreads) {
+    const int c = base + tid;
+    uint32_t key = 0;
+    bool in = c < NC;
+    if (in) key = chunk_key(score, c, NC, L, C);
+    const bool eq = in && key == theta;
+    const bool gt = in && key > theta;
+    // exclusive count of `eq` before this chunk
+    const uint32_t beq = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) warp_tot[0][warp] = __popc(beq);
+    __syncthreads();
+    uint32_t eq_before = carry[0] + __popc(beq & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) eq_before += warp_tot[0][w];
+    const bool keep = gt || (eq && eq_before < need_eq);
+    const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) warp_tot[1][warp] = __popc(bk);
+    __syncthreads();
+    uint32_t pos = carry[1] + __popc(bk & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += warp_tot[1][w];
+    if (keep && pos < (uint32_t)keff) idx[pos] = c;
+    __syncthreads();
+    if (tid == kSelThreads - 1) {
+      carry[0] = eq_before + (eq ? 1u : 0u);
+      carry[1] = pos + (keep ? 1u : 0u);
+    }
+    __syncthreads();
+  }
+  if (tid == 0) *n_selected = keff;
+}
+
+struct GatherArgs {
+  const __nv_bfloat16* src[2];
+  __nv_bfloat16* dst[2];
+  const int32_t* idx;
+  const int32_t* n_selected;
+  int32_t* n_tokens_out;
+  int32_t* status;
+  int n_layers, H, D, L, C, NC, max_selected, sub;
+  long long s_layer, s_l, s_h;
+};
+
+__global__ void __launch_bounds__(256) gather_kernel(const __grid_constant__ GatherArgs g) {
+  const int i = blockIdx.x / g.sub;                  // which selected chunk
+  const int part = blockIdx.x - i * g.sub;           // which slice of its tokens
+  const int layer = blockIdx.y;
+  const int which = blockIdx.z;                      // 0 = K, 1 = V
+  int nsel = *g.n_selected;
+  nsel = max(0, min(nsel, g.max_selected));
+  if (blockIdx.x == 0 && layer == 0 && which == 0 && threadIdx.x == 0) {
+    int ntok = 0;
+    if (nsel > 0) {
+      const int last = g.idx[nsel - 1];
+      if (last >= 0 && last < g.NC) ntok = (nsel - 1) * g.C + min(g.C, g.L - last * g.C);
+    }
+    *g.n_tokens_out = ntok;
+  }
+  if (i >= nsel) return;
+  const int c = g.idx[i];
+  if (c < 0 || c >= g.NC) {
+    if (threadIdx.x == 0 && part == 0) spx_raise(g.status, SPECEXT_ERR_INVALID_ARG);
+    return;
+  }
+  const int len = min(g.C, g.L - c * g.C);
+  const int tok_per_part = (g.C + g.sub - 1) / g.sub;
+  const int o_lo = part * tok_per_part, o_hi = min(len, o_lo + tok_per_part);
+  const int vpr = g.D / 8;                            // 16-byte vectors per head row
+  const int vpt = g.H * vpr;                          // per token
+  const __nv_bfloat16* src = g.src[which] + (long long)layer * g.s_layer;
+  __nv_bfloat16* dst = g.dst[which] + ((long long)layer * g.max_selected * g.C + (long long)i * g.C) * g.H * g.D;
+  const int nvec = max(0, o_hi - o_lo) * vpt;
+  for (int v = threadIdx.x; v < nvec; v += 256) {
+    const int o = o_lo + v / vpt;
+    const int w = v - (v / vpt) * vpt;
+    const int hh = w / vpr, dv = w - hh * vpr;
+    const uint4 x = *reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o) * g.s_l + (long long)hh * g.s_h + dv * 8);
+    *reinterpret_cast<uint4*>(dst + ((long long)o * g.H + hh) * g.D + dv * 8) = x;
+  }
+}
+
+}  // namespace
+
+cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
+                              int32_t* n_selected, cudaStream_t st) {
+  select_kernel<<<1, kSelThreads, 0, st>>>(score_row, NC, L, C, k, idx, n_selected);
+  return cudaGetLastError();
+}
+
+cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
+                              long long s_layer, long long s_l, long long s_h, const int32_t* idx,
+                              const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
+                              int32_t* n_tokens_out, int32_t* status, cudaStream_t st) {
+  GatherArgs g;
+  g.src[0] = static_cast<const __nv_bfloat16*>(dK);
+  g.src[1] = static_cast<const __nv_bfloat16*>(dV);
+  g.dst[0] = static_cast<__nv_bfloat16*>(K_out);
+  g.dst[1] = static_cast<__nv_bfloat16*>(V_out);
+  g.idx = idx;
+  g.n_selected = n_selected;
+  g.n_tokens_out = n_tokens_out;
+  g.status = status;
+  g.n_layers = n_layers; g.H = H; g.D = D; g.L = L; g.C = C;
+  g.NC = (L + C - 1) / C;
+  g.max_selected = max_selected;
+  // aim for ~16 KB per CTA
+  const long long chunk_bytes = (long long)C * H * D * 2;
+  int sub = (int)((chunk_bytes + 16383) / 16384);
+  sub = max(1, min(sub, C));
+  g.sub = sub;
+  g.s_layer = s_layer; g.s_l = s_l; g.s_h = s_h;
+  const dim3 grid(max_selected * sub, n_layers, 2);
+  gather_kernel<<<grid, 256, 0, st>>>(g);
+  return cudaGetLastError();
+}

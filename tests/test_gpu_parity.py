@@ -1,0 +1,360 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 CPU oracle, element by element.
+
+Tolerances (bf16 inputs, fp32 accumulation): O max-abs error <= 1e-2; lse abs error <= 1e-3;
+chunk_score relative error <= 1e-3; selected chunk indices and gathered KV bit-exact, with the
+top-k set allowed to differ only where the oracle's k-th / (k+1)-th ranking keys are closer than
+1e-4 relative.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import specext_oracle as orc
+from paper_2505_20776_b200 import api, synth
+from paper_2505_20776_b200.hotpath import HotPath
+from tests.util import bf16_bits, f64, random_forest
+
+pytestmark = pytest.mark.gpu
+
+O_ATOL = 1e-2
+LSE_ATOL = 1e-3
+SCORE_RTOL = 1e-3
+NEAR_TIE = 1e-4
+
+
+def oracle_layer(t, parent, L, C, scale=None):
+    return orc.verify_attn(f64(t["Q"]), f64(t["K_prefix"][:L]), f64(t["V_prefix"][:L]), f64(t["K_tree"]),
+                           f64(t["V_tree"]), parent, C, scale)
+
+
+def to_dev(t, dev):
+    return {k: v.to(dev) for k, v in t.items()}
+
+
+def check_attn(hp, t_cpu, parent, L, C, want_score=True, scale=None):
+    """Runs the GPU attention on the given host tensors and compares against the oracle."""
+    dev = hp.device
+    t = to_dev(t_cpu, dev)
+    par = torch.from_numpy(np.asarray(parent, dtype=np.int32)).to(dev)
+    hp.verify_attn(t, par, L, want_score)
+    assert hp.read_status() == 0
+    O_ref, lse_ref, cs_ref = oracle_layer(t_cpu, parent, L, C, scale)
+    O = f64(hp.O)
+    lse = f64(hp.lse)
+    assert np.isfinite(O).all() and np.isfinite(lse).all()
+    assert np.abs(O - O_ref).max() <= O_ATOL
+    assert np.abs(lse - lse_ref).max() <= LSE_ATOL
+    if want_score and L > 0:
+        cs = f64(hp.chunk_score(L))
+        assert cs.shape == cs_ref.shape
+        assert np.isfinite(cs).all()
+        rel = np.abs(cs - cs_ref) / np.maximum(cs_ref, 1e-30)
+        assert rel.max() <= SCORE_RTOL, f"chunk_score rel err {rel.max():.3e}"
+    return O_ref, lse_ref, cs_ref
+
+
+def check_retrieval(hp, cs_ref, rows, L, C, k, draft_cpu):
+    """select + gather on the GPU's own scores vs the oracle's decision on the oracle's scores."""
+    dev = hp.device
+    dK, dV = draft_cpu
+    dKd, dVd = dK.to(dev), dV.to(dev)
+    NC = cs_ref.shape[1]
+    lens = orc.chunk_lengths(L, C)
+    for row in rows:
+        hp.select_chunks(row, L)
+        hp.gather_kv(dKd, dVd, L)
+        assert hp.read_status() == 0
+        nsel = int(hp.n_selected.item())
+        keff = min(k, NC)
+        assert nsel == keff
+        idx = hp.idx[:nsel].cpu().numpy()
+        assert np.all(np.diff(idx) > 0) and idx.min() >= 0 and idx.max() < NC
+        # the oracle's ranking, in fp64 on its own scores
+        ref_idx = orc.select_chunks(cs_ref[row], L, C, k, key_dtype=np.float64)
+        if set(idx.tolist()) != set(ref_idx.tolist()):
+            key = cs_ref[row] / lens
+            srt = np.sort(key)[::-1]
+            gap = (srt[keff - 1] - srt[keff]) / srt[keff - 1] if keff < NC else np.inf
+            diff = set(idx.tolist()) ^ set(ref_idx.tolist())
+            # only chunks within the near-tie band around the k-th key may differ
+            assert gap < NEAR_TIE, f"top-k sets differ with a clear gap {gap:.3e}"
+            for c in diff:
+                assert abs(key[c] - srt[keff - 1]) / srt[keff - 1] < NEAR_TIE
+        # gather: bit-exact against the oracle's gather for the indices the GPU chose
+        Kr, Vr, ntok = orc.gather_kv(dK.view(torch.int16).numpy(), dV.view(torch.int16).numpy(), idx, L, C)
+        assert int(hp.n_tokens.item()) == ntok
+        np.testing.assert_array_equal(bf16_bits(hp.K_compact)[:, :ntok], Kr)
+        np.testing.assert_array_equal(bf16_bits(hp.V_compact)[:, :ntok], Vr)
+
+
+def check_select_bit_exact(hp, score_row_f32, L, C, k):
+    """The same fp32 score row on both sides: indices must be identical."""
+    dev = hp.device
+    NC = len(score_row_f32)
+    cs = hp.chunk_score(L)
+    cs.zero_()
+    cs[0] = torch.from_numpy(score_row_f32).to(dev)
+    hp.select_chunks(0, L)
+    assert hp.read_status() == 0
+    nsel = int(hp.n_selected.item())
+    want = orc.select_chunks(score_row_f32, L, C, k)
+    assert nsel == len(want) == min(k, NC)
+    np.testing.assert_array_equal(hp.idx[:nsel].cpu().numpy(), want)
+
+
+def make_hp(w, dev, max_prefix=None, k=None, scale=0.0):
+    return HotPath(w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_tree, w.chunk_size, k or w.top_k,
+                   max_prefix or (w.capacity or w.prefix_len), device=dev, softmax_scale=scale)
+
+
+# ---------------------------------------------------------------------------------------------
+# the five workload configurations
+
+
+def test_c0_tiny(cuda_device):
+    w = synth.WORKLOADS["c0"]
+    hp = make_hp(w, cuda_device)
+    t = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, w.prefix_len, w.chunk_size)
+    check_retrieval(hp, cs, range(w.n_tree), w.prefix_len, w.chunk_size, w.top_k, synth.make_draft_kv(w))
+
+
+@pytest.mark.parametrize("background", ["graded", "flat"])
+def test_c1_llama8b_4k(cuda_device, background):
+    w = synth.WORKLOADS["c1"]
+    hp = make_hp(w, cuda_device)
+    t = synth.make_layer(w, background=background)
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, w.prefix_len, w.chunk_size)
+    check_retrieval(hp, cs, range(w.n_tree), w.prefix_len, w.chunk_size, w.top_k, synth.make_draft_kv(w))
+    _, needles = synth.needle_profile(w, w.n_chunks, background)
+    hp.select_chunks(37, w.prefix_len)
+    assert set(needles.tolist()) <= set(hp.idx.cpu().numpy().tolist())
+
+
+@pytest.mark.parametrize("layer", [0, 15, 31])
+def test_c2_llama8b_16k_layers(cuda_device, layer):
+    w = synth.WORKLOADS["c2"]
+    hp = make_hp(w, cuda_device)
+    t = synth.make_layer(w, layer=layer)
+    parent = synth.make_tree(w)
+    want = layer == 31
+    _, _, cs = check_attn(hp, t, parent, w.prefix_len, w.chunk_size, want_score=want)
+    if want:
+        check_retrieval(hp, cs, [0, 37, 59], w.prefix_len, w.chunk_size, w.top_k, synth.make_draft_kv(w))
+
+
+def test_c3_growth_sweep_in_place(cuda_device):
+    """One KV buffer of the sweep's capacity; bytes beyond the current length are NaN and must not
+    influence any output.  Lengths are the sweep's, capped so the oracle stays within seconds, plus
+    ragged ones."""
+    w = synth.WORKLOADS["c3"]
+    cap = 8192 + 128
+    dev = cuda_device
+    hp = make_hp(w, dev, max_prefix=cap)
+    full = synth.make_layer(w, capacity=cap)
+    draft = synth.make_draft_kv(w, capacity=cap)
+    parent = synth.make_tree(w)
+    for L in (1024, 2048, 4096, 8192, 1000, 4097, 8192 + 31):
+        t = {k: v.clone() for k, v in full.items()}
+        t["K_prefix"][L:] = float("nan")
+        t["V_prefix"][L:] = float("nan")
+        _, _, cs = check_attn(hp, t, parent, L, w.chunk_size)
+        check_retrieval(hp, cs, [37], L, w.chunk_size, w.top_k, draft)
+
+
+def test_c3_long_lengths_sampled_rows(cuda_device):
+    """16K and 32K of the sweep: the oracle checks a sample of query heads (all nodes) per length."""
+    w = synth.WORKLOADS["c3"]
+    dev = cuda_device
+    parent = synth.make_tree(w)
+    full = synth.make_layer(w, capacity=32768)
+    hp = make_hp(w, dev, max_prefix=32768)
+    for L in (16384, 32768):
+        t = to_dev(full, dev)
+        par = torch.from_numpy(parent).to(dev)
+        hp.verify_attn(t, par, L, True)
+        assert hp.read_status() == 0
+        O, lse = f64(hp.O), f64(hp.lse)
+        G = w.group
+        for h in (0, 13, 31):
+            g = h // G
+            sub = {"Q": full["Q"][:, h:h + 1], "K_prefix": full["K_prefix"][:L, g:g + 1],
+                   "V_prefix": full["V_prefix"][:L, g:g + 1], "K_tree": full["K_tree"][:, g:g + 1],
+                   "V_tree": full["V_tree"][:, g:g + 1]}
+            O_ref, lse_ref, _ = oracle_layer(sub, parent, L, w.chunk_size)
+            assert np.abs(O[:, h] - O_ref[:, 0]).max() <= O_ATOL
+            assert np.abs(lse[h] - lse_ref[0]).max() <= LSE_ATOL
+        # properties that hold at any size: scores are non-negative and each row sums to <= 1
+        cs = f64(hp.chunk_score(L))
+        assert (cs >= 0).all() and (cs.sum(1) <= 1 + 1e-4).all() and (cs.sum(1) > 0.5).all()
+
+
+def test_c4_70b_class(cuda_device):
+    w = synth.WORKLOADS["c4"]
+    hp = make_hp(w, cuda_device)
+    t = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, w.prefix_len, w.chunk_size)
+    check_retrieval(hp, cs, [0, 37], w.prefix_len, w.chunk_size, w.top_k, synth.make_draft_kv(w))
+
+
+# ---------------------------------------------------------------------------------------------
+# edge cases
+
+
+def _small(Hq, Hkv, D, L, T, C, k=4, tree="uniform", values="normal", seed=7):
+    return synth.Workload("edge", Hq, Hkv, D, L, T, C, k, tree, values, seed=seed)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,L,T,C", [
+    (4, 1, 64, 0, 1, 32),        # empty prefix, single node: O = V_tree[0]
+    (4, 2, 64, 0, 9, 32),        # empty prefix, tree only
+    (4, 4, 128, 1, 1, 1),        # two keys, chunk size 1
+    (8, 2, 128, 127, 13, 16),    # one ragged key tile
+    (8, 2, 128, 129, 13, 16),    # a full tile and a one-key tail
+    (2, 2, 64, 300, 64, 128),    # MHA (G = 1), maximum tree, maximum chunk size
+    (64, 1, 128, 513, 5, 64),    # G = 64: 320 stacked rows -> two row blocks
+    (16, 8, 128, 2048 + 77, 60, 8),
+])
+def test_edge_shapes(cuda_device, Hq, Hkv, D, L, T, C):
+    w = _small(Hq, Hkv, D, L, T, C)
+    hp = make_hp(w, cuda_device, max_prefix=max(L, 1))
+    t = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, L, C)
+    if L > 0:
+        check_retrieval(hp, cs, [T - 1], L, C, w.top_k, synth.make_draft_kv(w))
+    else:
+        hp.select_chunks(0, 0)
+        assert hp.read_status() == 0 and int(hp.n_selected.item()) == 0
+
+
+def test_single_key_returns_value_exactly(cuda_device):
+    w = _small(4, 1, 64, 0, 1, 32)
+    hp = make_hp(w, cuda_device, max_prefix=1)
+    t = synth.make_layer(w)
+    dev = cuda_device
+    hp.verify_attn(to_dev(t, dev), torch.tensor([-1], dtype=torch.int32, device=dev), 0, False)
+    assert hp.read_status() == 0
+    for h in range(4):
+        assert torch.equal(hp.O[0, h].cpu(), t["V_tree"][0, 0])
+
+
+def test_chain_tree_and_explicit_scale(cuda_device):
+    w = _small(8, 2, 128, 500, 33, 32, tree="chain")
+    hp = make_hp(w, cuda_device, scale=0.05)
+    t = synth.make_layer(w)
+    check_attn(hp, t, synth.make_tree(w), 500, 32, scale=0.05)
+
+
+def test_zero_query_gives_first_k_chunks(cuda_device):
+    w = _small(8, 2, 128, 1000, 7, 32, k=5)
+    hp = make_hp(w, cuda_device)
+    t = synth.make_layer(w)
+    t["Q"].zero_()
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, 1000, 32)
+    # full chunks have exactly equal mass on the GPU too (same arithmetic for each), so ties
+    # resolve to the lowest indices
+    hp.select_chunks(0, 1000)
+    np.testing.assert_array_equal(hp.idx[:5].cpu().numpy(), np.arange(5))
+
+
+def test_strided_inputs(cuda_device):
+    """K/V views into a wider cache (extra heads, padded rows) must give the same result."""
+    w = _small(8, 2, 128, 700, 11, 32)
+    dev = cuda_device
+    hp = make_hp(w, dev)
+    t = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    O_ref, lse_ref, _ = oracle_layer(t, parent, 700, 32)
+    big_k = torch.full((800, 5, 136), float("nan"), dtype=torch.bfloat16, device=dev)
+    big_v = torch.full((800, 5, 136), float("nan"), dtype=torch.bfloat16, device=dev)
+    big_k[:700, 1:3, :128] = t["K_prefix"].to(dev)
+    big_v[:700, 1:3, :128] = t["V_prefix"].to(dev)
+    td = to_dev(t, dev)
+    td["K_prefix"] = big_k[:, 1:3, :128]
+    td["V_prefix"] = big_v[:, 1:3, :128]
+    qbig = torch.zeros(11, 8, 256, dtype=torch.bfloat16, device=dev)
+    qbig[:, :, :128] = td["Q"]
+    td["Q"] = qbig[:, :, :128]
+    hp.verify_attn(td, torch.from_numpy(parent).to(dev), 700, True)
+    assert hp.read_status() == 0
+    assert np.abs(f64(hp.O) - O_ref).max() <= O_ATOL
+    assert np.abs(f64(hp.lse) - lse_ref).max() <= LSE_ATOL
+
+
+def test_select_bit_exact_on_given_scores(cuda_device):
+    rng = np.random.default_rng(5)
+    for NC, C, tail, k in [(1, 32, 0, 1), (5, 32, 3, 3), (512, 32, 0, 32), (1024, 32, 7, 32), (2500, 8, 1, 300),
+                           (40000, 4, 2, 1000), (64, 32, 0, 64), (64, 32, 0, 100)]:
+        L = NC * C - tail
+        w = _small(4, 1, 64, L, 2, C, k=k)
+        hp = HotPath(4, 1, 64, 2, C, k, L, device=cuda_device)
+        score = rng.random(NC).astype(np.float32)
+        check_select_bit_exact(hp, score, L, C, k)
+        tied = (np.round(score * 4) / 4).astype(np.float32)            # many exact ties
+        check_select_bit_exact(hp, tied, L, C, k)
+        check_select_bit_exact(hp, np.full(NC, 0.25, dtype=np.float32), L, C, k)
+
+
+def test_bad_tree_sets_status(cuda_device):
+    w = _small(4, 1, 64, 64, 4, 32)
+    dev = cuda_device
+    hp = make_hp(w, dev)
+    t = to_dev(synth.make_layer(w), dev)
+    for bad in ([0, 0, 1, 2], [-1, 2, 0, 1], [-2, 0, 1, 2]):
+        hp.status.zero_()
+        hp.verify_attn(t, torch.tensor(bad, dtype=torch.int32, device=dev), 64, False)
+        assert api.status_bits(hp.read_status()) == ("BAD_TREE",)
+    hp.status.zero_()
+
+
+def test_host_validation(cuda_device):
+    w = _small(4, 1, 64, 64, 4, 32)
+    dev = cuda_device
+    hp = make_hp(w, dev)
+    t = to_dev(synth.make_layer(w), dev)
+    par = torch.tensor([-1, 0, 1, 2], dtype=torch.int32, device=dev)
+    d = api.make_attn_desc(t["Q"], t["K_prefix"], t["K_tree"], hp.O, 64, 32)
+    ws = torch.empty(api.specext_verify_attn_workspace(d), dtype=torch.uint8, device=dev)
+
+    def call(desc, workspace=ws):
+        api.specext_verify_attn(desc, t["Q"], t["K_prefix"], t["V_prefix"], t["K_tree"], t["V_tree"], par, hp.O,
+                                hp.lse, None, workspace, hp.status)
+    call(d)
+    for field, value, code in [("head_dim", 96, 2), ("n_tree", 65, 2), ("chunk_size", 48, 2),
+                               ("n_kv_heads", 3, 1), ("kv_stride_l", 60, 1), ("prefix_len", -1, 1)]:
+        bad = api.AttnDesc.from_buffer_copy(d)
+        setattr(bad, field, value)
+        with pytest.raises(api.SpecextError) as e:
+            call(bad)
+        assert e.value.code == code
+    with pytest.raises(api.SpecextError) as e:
+        call(d, ws[:128])
+    assert e.value.code == 3
+    with pytest.raises(api.SpecextError):
+        api.specext_select_chunks(hp.chunk_score(64), 9, 64, 32, 4, hp.idx, hp.n_selected, hp.status)
+    with pytest.raises(api.SpecextError):
+        api.specext_select_chunks(hp.chunk_score(64), 0, 64, 32, 0, hp.idx, hp.n_selected, hp.status)
+    assert hp.read_status() == 0
+
+
+def test_determinism_run_to_run(cuda_device):
+    w = synth.WORKLOADS["c1"]
+    dev = cuda_device
+    hp = make_hp(w, dev)
+    t = to_dev(synth.make_layer(w), dev)
+    par = torch.from_numpy(synth.make_tree(w)).to(dev)
+    outs = []
+    for _ in range(3):
+        hp.verify_attn(t, par, w.prefix_len, True)
+        torch.cuda.synchronize()
+        outs.append((hp.O.clone(), hp.lse.clone(), hp.chunk_score(w.prefix_len).clone()))
+    for o in outs[1:]:
+        for a, b in zip(o, outs[0]):
+            assert torch.equal(a, b)
