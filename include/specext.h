@@ -149,6 +149,17 @@ const char* specext_status_string(int status);
 /* Number of kernels the library has launched in this process (all calls, all streams). */
 int64_t specext_launch_count(void);
 
+/*
+ * Process-wide tuning and cross-check switches (the paper has no counterpart).
+ *   attn_kernel       : 0 or 2 = tensor-core (tcgen05) attention kernel, the default;
+ *                       1 = the CUDA-core kernel, an independent on-device cross-check.
+ *   min_tiles_per_cta : lower bound on the 128-key tiles one CTA processes (> 0 to change; fewer,
+ *                       longer splits mean fewer partial results to merge).  Changes the
+ *                       workspace size, so set it before querying specext_verify_attn_workspace.
+ * Not thread-safe with respect to concurrent calls of the library.
+ */
+int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta);
+
 #ifdef __cplusplus
 }
 #endif

@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
     L.specext_status_string.argtypes = [ctypes.c_int]
     L.specext_launch_count.restype = i64
     L.specext_launch_count.argtypes = []
+    L.specext_set_tuning.restype = ctypes.c_int
+    L.specext_set_tuning.argtypes = [i32, i32]
     _LIB = L
     return L
 
@@ -178,6 +180,10 @@ def specext_read_status(device_status: torch.Tensor) -> int:
 
 def specext_launch_count() -> int:
     return int(lib().specext_launch_count())
+
+
+def specext_set_tuning(attn_kernel: int = 0, min_tiles_per_cta: int = 0) -> None:
+    _check(lib().specext_set_tuning(int(attn_kernel), int(min_tiles_per_cta)), "specext_set_tuning")
 
 
 def status_bits(bits: int) -> Tuple[str, ...]:

@@ -137,7 +137,7 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int n = 0;
-  cudaError_t e = spx_launch_attn_simt(a, st, &n);
+  cudaError_t e = g_attn_kernel.load() == 1 ? spx_launch_attn_simt(a, st, &n) : spx_launch_attn_tc(a, st, &n);
   if (e == cudaSuccess) e = spx_launch_merge(a, st, &n);
   g_launches.fetch_add(n);
   if (e != cudaSuccess) {
@@ -228,5 +228,12 @@ const char* specext_status_string(int status) {
 }
 
 int64_t specext_launch_count(void) { return g_launches.load(); }
+
+int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta) {
+  if (attn_kernel < 0 || attn_kernel > 2 || min_tiles_per_cta < 0) return SPECEXT_ERR_INVALID_ARG;
+  g_attn_kernel.store(attn_kernel);
+  if (min_tiles_per_cta > 0) g_min_units.store(min_tiles_per_cta);
+  return SPECEXT_OK;
+}
 
 }  // extern "C"

@@ -1,0 +1,482 @@
+// Hybrid Tree Attention on the sm_100a tensor cores: split-over-KV partial attention of the stacked
+// (query head x tree node) rows of one KV head against 128-key tiles of the prefix and the tree.
+//
+// CTA = 10 warps, one CTA per SM, persistent over its range of (problem, key tile) units:
+//   warp 0      TMA producer: Q tile of the segment (once), then K and V tiles into a shared-memory
+//               ring (128-byte swizzle, 64-element column blocks), completion on mbarriers.
+//   warp 1      MMA issuer: S = Q K^T (both operands K-major in shared memory) into tensor memory,
+//               O += P V with P read from tensor memory and V as an MN-major shared-memory operand.
+//   warps 2-5   softmax of row tile 0 (one thread per query row), warps 6-9 of row tile 1:
+//               tcgen05.ld of S, running maximum with lazy rescaling of O, exp2 in fp32, row and
+//               per-chunk sums from the unrounded exponentials, P rounded to bf16 back into the
+//               columns S occupied.
+// Tensor memory (512 columns): O tile 0 | O tile 1 | S/P tile 0 | S/P tile 1, 128 columns each.
+// The two row tiles are interleaved on the tensor pipe (S0 S1 | PV0 S0' PV1 S1' | ...) so that
+// the softmax of one tile runs under the MMAs of the other.
+//
+// Every mbarrier wait is bounded; on expiry the CTA raises SPECEXT_ERR_TIMEOUT, drains its copies
+// and MMAs (bounded again), frees tensor memory and returns.
+#include "common.cuh"
+#include "sm100.cuh"
+
+using namespace sm100;
+
+struct TcMaps {
+  CUtensorMap q, kp, vp, kt, vt;
+};
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kSubTileBytes = 128 * 128;        // 128 rows x 64 bf16
+constexpr float kRescaleThreshold = 8.0f;       // log2 units
+
+template <int D>
+struct Cfg {
+  static constexpr int DS = D / 64;                           // 64-element column blocks
+  static constexpr int kStageBytes = DS * kSubTileBytes;      // one K or V tile
+  static constexpr int kQBytes = 2 * DS * kSubTileBytes;      // two row tiles
+  static constexpr int kStages = D == 128 ? 5 : 8;
+  static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
+  static constexpr int kSmemBytes = kBarOffset + 1024 + 1024; // + control block + alignment slack
+};
+
+struct Ctrl {
+  uint64_t q_full, q_free, drain;
+  uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+  uint64_t kv_full[8], kv_empty[8];
+  unsigned long long anc[64];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int D, bool SCORE>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMaps maps) {
+  using C = Cfg<D>;
+  constexpr int DS = C::DS;
+  constexpr int NS = C::kStages;
+  const AttnPlan& p = a.plan;
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  unsigned char* Qs = base;
+  unsigned char* ring = base + C::kQBytes;
+  Ctrl* ctl = reinterpret_cast<Ctrl*>(base + C::kBarOffset);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_mt = p.RB / 128;
+  const int cta = blockIdx.x;
+  const int unit_lo = spx_unit_start(p, cta), unit_hi = spx_unit_start(p, cta + 1);
+
+  if (tid == 0) {
+    mbar_init(&ctl->q_full, 1);
+    mbar_init(&ctl->q_free, 1);
+    mbar_init(&ctl->drain, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ctl->s_full[i], 1);
+      mbar_init(&ctl->p_full[i], 128);
+      mbar_init(&ctl->o_done[i], 1);
+      mbar_init(&ctl->o_free[i], 128);
+    }
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(&ctl->kv_full[i], 1);
+      mbar_init(&ctl->kv_empty[i], 1);
+    }
+    ctl->abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&maps.q);
+    prefetch_tensormap(&maps.kp);
+    prefetch_tensormap(&maps.vp);
+    prefetch_tensormap(&maps.kt);
+    prefetch_tensormap(&maps.vt);
+  }
+  spx_build_ancestors(a.parent, p.T, ctl->anc, cta == 0 ? a.status : nullptr);
+  if (warp == 1) {
+    tmem_alloc(&ctl->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+  bool ok = true;
+
+  if (warp == 0) {
+    // ================================ TMA producer ==========================================
+    if (lane == 0) {
+      uint32_t kvp = 0;
+      int seg = 0;
+      bool q_armed = false;
+      for (int u = unit_lo; u < unit_hi && ok;) {
+        const int prob = u / p.UPP;
+        const int tile_lo = u - prob * p.UPP;
+        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+        const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+        if (seg > 0) ok = mbar_wait(&ctl->q_free, (seg - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&ctl->q_full, n_mt * DS * kSubTileBytes);
+        q_armed = true;
+        for (int mt = 0; mt < n_mt; ++mt)
+          for (int ds = 0; ds < DS; ++ds)
+            tma_load_3d(Qs + (mt * DS + ds) * kSubTileBytes, &maps.q, &ctl->q_full, ds * 64, g * p.G,
+                        (rblk * n_mt + mt) * (128 / p.G));
+        for (int tile = tile_lo; tile < tile_hi && ok; ++tile) {
+          const bool is_tree = tile == p.TPH;
+          for (int which = 0; which < 2; ++which) {
+            const int stage = kvp % NS;
+            ok = mbar_wait(&ctl->kv_empty[stage], ((kvp / NS) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&ctl->kv_full[stage], C::kStageBytes);
+            const CUtensorMap* m = is_tree ? (which ? &maps.vt : &maps.kt) : (which ? &maps.vp : &maps.kp);
+            for (int ds = 0; ds < DS; ++ds)
+              tma_load_3d(ring + stage * C::kStageBytes + ds * kSubTileBytes, m, &ctl->kv_full[stage], ds * 64, g,
+                          is_tree ? 0 : tile * SPX_TILE_KEYS);
+            ++kvp;
+          }
+        }
+        u += tile_hi - tile_lo;
+        ++seg;
+      }
+      if (!ok) {
+        // give the copies already issued a bounded chance to land before the CTA's memory is released
+        const uint32_t lo = kvp > (uint32_t)NS ? kvp - NS : 0;
+        for (uint32_t f = lo; f < kvp; ++f)
+          for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&ctl->kv_full[f % NS], (f / NS) & 1); ++spin) {}
+        if (q_armed)
+          for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&ctl->q_full, (seg > 0 ? seg - 1 : 0) & 1); ++spin) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ============================================
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16_f32(128, SPX_TILE_KEYS, false, false);
+      const uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
+      const uint32_t q_addr = smem_u32(Qs), ring_addr = smem_u32(ring);
+      uint32_t kvc = 0, it = 0;
+      int seg = 0;
+
+      auto issue_s = [&](int mt, int stage) {
+        const uint32_t kb = ring_addr + stage * C::kStageBytes;
+        const uint32_t qb = q_addr + mt * DS * kSubTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * kSubTileBytes + (kk & 3) * 32;
+          mma_ss(tmem + 256 + mt * 128, smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
+                 idesc_s, kk > 0);
+        }
+        mma_commit(&ctl->s_full[mt]);
+      };
+      auto issue_pv = [&](int mt, int stage, bool accumulate) {
+        const uint32_t vb = ring_addr + stage * C::kStageBytes;
+#pragma unroll
+        for (int kk = 0; kk < SPX_TILE_KEYS / 16; ++kk)
+          mma_ts(tmem + mt * 128, tmem + 256 + mt * 128 + kk * 8,
+                 smem_desc_sw128(vb + kk * 2048, kSubTileBytes, 1024), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
+      };
+
+      for (int u = unit_lo; u < unit_hi && ok;) {
+        const int prob = u / p.UPP;
+        const int tile_lo = u - prob * p.UPP;
+        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+        const int n = tile_hi - tile_lo;
+        ok = mbar_wait(&ctl->q_full, seg & 1, abort_flag);
+        if (!ok) break;
+        {
+          const int ks = kvc % NS;
+          ok = mbar_wait(&ctl->kv_full[ks], (kvc / NS) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          for (int mt = 0; mt < n_mt; ++mt) issue_s(mt, ks);
+          mma_commit(&ctl->kv_empty[ks]);
+          ++kvc;
+        }
+        for (int i = 0; i < n && ok; ++i) {
+          const bool has_next = i + 1 < n, last = !has_next;
+          const int vs = kvc % NS;
+          const uint32_t vph = (kvc / NS) & 1;
+          ++kvc;
+          const int ks = kvc % NS;
+          const uint32_t kph = (kvc / NS) & 1;
+          ok = mbar_wait(&ctl->kv_full[vs], vph, abort_flag);
+          for (int mt = 0; mt < n_mt && ok; ++mt) {
+            ok = mbar_wait(&ctl->p_full[mt], it & 1, abort_flag);
+            if (ok && i == 0 && seg > 0) ok = mbar_wait(&ctl->o_free[mt], (seg - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(mt, vs, i > 0);
+            if (last) mma_commit(&ctl->o_done[mt]);
+            if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[vs]);
+            if (has_next) {
+              if (mt == 0) {
+                ok = mbar_wait(&ctl->kv_full[ks], kph, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+              }
+              issue_s(mt, ks);
+              if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[ks]);
+            }
+          }
+          if (has_next) ++kvc;
+          ++it;
+        }
+        if (ok) mma_commit(&ctl->q_free);
+        u += n;
+        ++seg;
+      }
+      // drain: all MMAs issued so far must have completed before tensor memory is released
+      mma_commit(&ctl->drain);
+      for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(&ctl->drain, 0); ++spin) {}
+    }
+  } else {
+    // ================================ softmax warps =========================================
+    const int mt = (warp - 2) >> 2;
+    if (mt < n_mt) {
+      const int quarter = warp & 3;
+      const int row_t = quarter * 32 + lane;
+      const int rr = mt * 128 + row_t;
+      const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+      const uint32_t s_addr = tmem + lane_addr + 256 + mt * 128;
+      const uint32_t o_addr = tmem + lane_addr + mt * 128;
+      const float scale2 = p.scale2;
+      uint32_t it = 0;
+      int seg = 0;
+      for (int u = unit_lo; u < unit_hi && ok;) {
+        const int prob = u / p.UPP;
+        const int tile_lo = u - prob * p.UPP;
+        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+        const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+        const int r = rblk * p.RB + rr;
+        const bool valid = r < p.rows;
+        const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
+        float m_used = -INFINITY, l = 0.f;
+
+        for (int tile = tile_lo; tile < tile_hi; ++tile, ++it) {
+          const bool is_tree = tile == p.TPH;
+          const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
+          const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
+          unsigned long long vis_lo = ~0ull, vis_hi = ~0ull;
+          if (is_tree) {
+            vis_lo = tree_mask;
+            vis_hi = 0ull;
+          } else if (need_mask) {
+            vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
+            vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);
+          }
+          ok = mbar_wait(&ctl->s_full[mt], it & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+
+          // pass 1: maximum of the visible raw scores of this row
+          float tmax = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t v[32];
+            tmem_ld32(s_addr + c * 32, v);
+            tmem_wait_ld();
+            if (need_mask) {
+              const uint32_t bits = static_cast<uint32_t>((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                tmax = fmaxf(tmax, ((bits >> j) & 1u) ? __uint_as_float(v[j]) : -INFINITY);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) tmax = fmaxf(tmax, __uint_as_float(v[j]));
+            }
+          }
+          const float m_tile = tmax * scale2;
+          float alpha = 1.f;
+          bool rescale = false;
+          if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
+            alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
+            rescale = tile > tile_lo;
+            m_used = m_tile;
+            l *= alpha;
+          }
+          if (__any_sync(0xffffffffu, rescale)) {
+            // S(tile) has been committed after PV(tile-1), so O is complete and not being written
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t v[32];
+              tmem_ld32(o_addr + c * 32, v);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+              tmem_st32(o_addr + c * 32, v);
+            }
+          }
+
+          // pass 2: exponentials against the reference maximum, sums, P in bf16 back to tensor memory
+          const float neg_m = -m_used;
+          const bool score = SCORE && !is_tree;
+          float* mass = nullptr;
+          if (score) {
+            const long long rowbase = ((long long)prob * p.TPH + tile) * p.RB + rr;
+            mass = a.ws + p.off_mass + rowbase * p.CPT;
+            a.ws[p.off_mref + rowbase] = m_used;
+          }
+          float csum = 0.f;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t v[32];
+            tmem_ld32(s_addr + c * 32, v);
+            tmem_wait_ld();
+            const uint32_t bits = need_mask ? static_cast<uint32_t>((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32))
+                                            : 0xffffffffu;
+            float pr[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              float x = fmaf(__uint_as_float(v[j]), scale2, neg_m);
+              if (need_mask) x = ((bits >> j) & 1u) ? x : -INFINITY;
+              pr[j] = ex2_approx(x);
+            }
+            float gs0 = 0.f, gs1 = 0.f, gs2 = 0.f, gs3 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              gs0 += pr[j];
+              gs1 += pr[j + 1];
+              gs2 += pr[j + 2];
+              gs3 += pr[j + 3];
+            }
+            const float gs = (gs0 + gs1) + (gs2 + gs3);
+            l += gs;
+            if (score) {
+              if (p.C >= 32) {
+                csum += gs;
+                if ((((c + 1) * 32) & (p.C - 1)) == 0) {
+                  mass[((c + 1) * 32) / p.C - 1] = csum;
+                  csum = 0.f;
+                }
+              } else {
+                float acc = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  acc += pr[j];
+                  if (((j + 1) & (p.C - 1)) == 0) {
+                    mass[(c * 32 + j) / p.C] = acc;
+                    acc = 0.f;
+                  }
+                }
+              }
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(pr[2 * j], pr[2 * j + 1]);
+            tmem_st16(s_addr + c * 16, pk);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&ctl->p_full[mt]);
+        }
+        if (!ok) break;
+
+        // epilogue of the segment: unnormalised O, reference maximum and row sum to the partial slot
+        ok = mbar_wait(&ctl->o_done[mt], seg & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        {
+          const int slot = cta + prob;
+          float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + c * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 x = make_float4(__uint_as_float(v[q4 * 4]), __uint_as_float(v[q4 * 4 + 1]),
+                                           __uint_as_float(v[q4 * 4 + 2]), __uint_as_float(v[q4 * 4 + 3]));
+              *reinterpret_cast<float4*>(po + ((long long)(c * 8 + q4) * p.RB + rr) * 4) = x;
+            }
+          }
+          a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_used;
+          a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l;
+        }
+        tc_fence_before();
+        mbar_arrive(&ctl->o_free[mt]);
+        u += tile_hi - tile_lo;
+        ++seg;
+      }
+    }
+  }
+
+  if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 tensor [n2][n1][D] with element strides (s2, s1, 1); box = 64 x b1 x b2, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_map(CUtensorMap* m, const void* ptr, int D, long long n1, long long s1, long long n2, long long s2,
+                int b1, int b2) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)n1, (cuuint64_t)n2};
+  const cuuint64_t strides[2] = {(cuuint64_t)s1 * 2, (cuuint64_t)s2 * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)b1, (cuuint32_t)b2};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D, bool SCORE>
+cudaError_t launch(const AttnArgs& a, const TcMaps& maps, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<D>::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  attn_tc_kernel<D, SCORE><<<a.plan.n_cta, kThreads, Cfg<D>::kSmemBytes, st>>>(a, maps);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t spx_launch_attn_tc(const AttnArgs& a, cudaStream_t st, int* n_launches) {
+  const AttnPlan& p = a.plan;
+  TcMaps maps;
+  const int tok_per_tile = 128 / p.G;
+  bool ok = encode_map(&maps.q, a.Q, p.D, p.Hq, a.q_sh, p.T, a.q_st, p.G, tok_per_tile);
+  ok = ok && encode_map(&maps.kt, a.Kt, p.D, p.Hkv, a.tkv_sh, p.T, a.tkv_st, 1, SPX_TILE_KEYS);
+  ok = ok && encode_map(&maps.vt, a.Vt, p.D, p.Hkv, a.tkv_sh, p.T, a.tkv_st, 1, SPX_TILE_KEYS);
+  if (p.L > 0) {
+    ok = ok && encode_map(&maps.kp, a.Kp, p.D, p.Hkv, a.kv_sh, p.L, a.kv_sl, 1, SPX_TILE_KEYS);
+    ok = ok && encode_map(&maps.vp, a.Vp, p.D, p.Hkv, a.kv_sh, p.L, a.kv_sl, 1, SPX_TILE_KEYS);
+  } else {
+    maps.kp = maps.kt;
+    maps.vp = maps.vt;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+  cudaError_t e;
+  if (p.D == 128)
+    e = p.want_score ? launch<128, true>(a, maps, st) : launch<128, false>(a, maps, st);
+  else
+    e = p.want_score ? launch<64, true>(a, maps, st) : launch<64, false>(a, maps, st);
+  *n_launches += 1;
+  return e;
+}
