@@ -177,6 +177,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: run only this many layers per step (the JSON line says so; not a bench value)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -202,6 +204,9 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = synth.WORKLOADS[WORKLOAD]
+    if args.layers > 0:
+        import dataclasses
+        w = dataclasses.replace(w, n_layers=max(2, args.layers))
     NL, L = w.n_layers, w.prefix_len
     parent_np = synth.make_tree(w)
     parent = torch.from_numpy(parent_np).to(dev)
@@ -362,7 +367,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": WORKLOAD_DESC, "l2": "inputs larger than L2 (2.1 GB of K/V read per step)",
-                           "cuda_graph": graph is not None, "replicas": world},
+                           "cuda_graph": graph is not None, "replicas": world,
+                           **({"profiling_layers": NL} if args.layers > 0 else {})},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
                 "roofline": roof}
         if world == 1 and not args.no_cpu_baseline:

@@ -16,7 +16,10 @@ namespace {
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_attn_kernel{0};       // 0 = default, 1 = CUDA-core kernel, 2 = tensor-core kernel
-std::atomic<int> g_min_units{1};         // lower bound on key tiles per CTA (tuning knob)
+std::atomic<int> g_min_units{1};
+#ifdef SPX_TRACE
+long long* g_trace = nullptr;
+#endif         // lower bound on key tiles per CTA (tuning knob)
 
 int sm_count() {
   static std::atomic<int> cached{0};
@@ -134,6 +137,9 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
   a.kv_sl = desc->kv_stride_l; a.kv_sh = desc->kv_stride_h;
   a.tkv_st = desc->tkv_stride_t; a.tkv_sh = desc->tkv_stride_h;
   a.o_st = desc->o_stride_t; a.o_sh = desc->o_stride_h;
+#ifdef SPX_TRACE
+  a.trace = g_trace;
+#endif
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int n = 0;
@@ -228,6 +234,10 @@ const char* specext_status_string(int status) {
 }
 
 int64_t specext_launch_count(void) { return g_launches.load(); }
+
+#ifdef SPX_TRACE
+void specext_debug_set_trace(void* p) { g_trace = static_cast<long long*>(p); }
+#endif
 
 int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta) {
   if (attn_kernel < 0 || attn_kernel > 2 || min_tiles_per_cta < 0) return SPECEXT_ERR_INVALID_ARG;

@@ -1,15 +1,18 @@
 // Hybrid Tree Attention on the sm_100a tensor cores: split-over-KV partial attention of the stacked
 // (query head x tree node) rows of one KV head against 128-key tiles of the prefix and the tree.
 //
-// CTA = 10 warps, one CTA per SM, persistent over its range of (problem, key tile) units:
-//   warp 0      TMA producer: Q tile of the segment (once), then K and V tiles into a shared-memory
+// CTA = 3 warpgroups (384 threads), one CTA per SM, persistent over its range of (problem, key
+// tile) units:
+//   warps 0-3   softmax of row tile 0, one thread per query row: one tcgen05.ld of the whole
+//               128-column S row into registers, maximum with lazy rescaling of O, exp2 in fp32,
+//               row and per-chunk sums from the unrounded exponentials, P rounded to bf16 back into
+//               the columns S occupied.  Warps 4-7: the same for row tile 1.
+//   warp 8      TMA producer: Q tile of the segment (once), then K and V tiles into a shared-memory
 //               ring (128-byte swizzle, 64-element column blocks), completion on mbarriers.
-//   warp 1      MMA issuer: S = Q K^T (both operands K-major in shared memory) into tensor memory,
+//   warp 9      MMA issuer: S = Q K^T (both operands K-major in shared memory) into tensor memory,
 //               O += P V with P read from tensor memory and V as an MN-major shared-memory operand.
-//   warps 2-5   softmax of row tile 0 (one thread per query row), warps 6-9 of row tile 1:
-//               tcgen05.ld of S, running maximum with lazy rescaling of O, exp2 in fp32, row and
-//               per-chunk sums from the unrounded exponentials, P rounded to bf16 back into the
-//               columns S occupied.
+//   warps 10-11 build the ancestor masks of the tree, then idle.
+// Registers are moved from the third warpgroup to the two softmax warpgroups (setmaxnreg).
 // Tensor memory (512 columns): O tile 0 | O tile 1 | S/P tile 0 | S/P tile 1, 128 columns each.
 // The two row tiles are interleaved on the tensor pipe (S0 S1 | PV0 S0' PV1 S1' | ...) so that
 // the softmax of one tile runs under the MMAs of the other.
@@ -27,7 +30,15 @@ struct TcMaps {
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
+// Register hand-over between warpgroups.  The kernel is compiled for 168 registers per thread
+// (65536 / 384, rounded down to a multiple of 8); the third warpgroup shrinks to kRegsOther and
+// the two softmax warpgroups grow to kRegsSoftmax.  setmaxnreg.inc blocks until the registers it
+// asks for have been released inside the CTA's own allocation, so the release must cover the request.
+constexpr int kRegsLaunch = 168, kRegsOther = 64, kRegsSoftmax = 216;
+static_assert(128 * (kRegsLaunch - kRegsOther) >= 256 * (kRegsSoftmax - kRegsLaunch),
+              "setmaxnreg.inc would wait for registers that are never released");
 constexpr int kSubTileBytes = 128 * 128;        // 128 rows x 64 bf16
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
 
@@ -46,6 +57,7 @@ struct Ctrl {
   uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
   uint64_t kv_full[8], kv_empty[8];
   unsigned long long anc[64];
+  int parent[64];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -66,12 +78,15 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
   Ctrl* ctl = reinterpret_cast<Ctrl*>(base + C::kBarOffset);
   volatile int* abort_flag = &ctl->abort_flag;
 
+#ifdef SPX_TRACE
+  const long long spx_t_start = clock64();
+#endif
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_mt = p.RB / 128;
   const int cta = blockIdx.x;
   const int unit_lo = spx_unit_start(p, cta), unit_hi = spx_unit_start(p, cta + 1);
 
-  if (tid == 0) {
+  if (warp == kProducerWarp && lane == 0) {
     mbar_init(&ctl->q_full, 1);
     mbar_init(&ctl->q_free, 1);
     mbar_init(&ctl->drain, 1);
@@ -93,20 +108,14 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
     prefetch_tensormap(&maps.kt);
     prefetch_tensormap(&maps.vt);
   }
-  spx_build_ancestors(a.parent, p.T, ctl->anc, cta == 0 ? a.status : nullptr);
-  if (warp == 1) {
-    tmem_alloc(&ctl->tmem_base, 512);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = ctl->tmem_base;
+  __syncthreads();                       // barriers are initialised; the producer may start at once
   bool ok = true;
 
-  if (warp == 0) {
+  if (warp == kProducerWarp) {
     // ================================ TMA producer ==========================================
+    setmaxnreg_dec<kRegsOther>();
     if (lane == 0) {
+      SPX_EVT(0, 0);
       uint32_t kvp = 0;
       int seg = 0;
       bool q_armed = false;
@@ -134,6 +143,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             for (int ds = 0; ds < DS; ++ds)
               tma_load_3d(ring + stage * C::kStageBytes + ds * kSubTileBytes, m, &ctl->kv_full[stage], ds * 64, g,
                           is_tree ? 0 : tile * SPX_TILE_KEYS);
+            SPX_EVT(0, 1 + kvp);
             ++kvp;
           }
         }
@@ -149,255 +159,309 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           for (int spin = 0; spin < (1 << 20) && !mbar_try_wait(&ctl->q_full, (seg > 0 ? seg - 1 : 0) & 1); ++spin) {}
       }
     }
-  } else if (warp == 1) {
-    // ================================ MMA issuer ============================================
-    if (lane == 0) {
-      const uint32_t idesc_s = idesc_bf16_f32(128, SPX_TILE_KEYS, false, false);
-      const uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
-      const uint32_t q_addr = smem_u32(Qs), ring_addr = smem_u32(ring);
-      uint32_t kvc = 0, it = 0;
-      int seg = 0;
-
-      auto issue_s = [&](int mt, int stage) {
-        const uint32_t kb = ring_addr + stage * C::kStageBytes;
-        const uint32_t qb = q_addr + mt * DS * kSubTileBytes;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * kSubTileBytes + (kk & 3) * 32;
-          mma_ss(tmem + 256 + mt * 128, smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
-                 idesc_s, kk > 0);
+  } else {
+    // tensor memory (MMA warp) and ancestor masks (warps 10, 11), then everybody but the producer meets
+    if (warp == kMmaWarp) {
+      tmem_alloc(&ctl->tmem_base, 512);
+      tmem_relinquish();
+    } else if (warp > kMmaWarp) {
+      const int t = tid - (kMmaWarp + 1) * 32;                  // 0..63
+      ctl->parent[t] = t < p.T ? a.parent[t] : -1;
+      named_bar_sync(2, 64);
+      unsigned long long m = 0;
+      if (t < p.T) {
+        int u = t;
+        for (int step = 0; step <= p.T && u >= 0; ++step) {
+          m |= 1ull << u;
+          const int pu = ctl->parent[u];
+          if (pu < -1 || pu >= u) {
+            if (cta == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
+            break;
+          }
+          u = pu;
         }
-        mma_commit(&ctl->s_full[mt]);
-      };
-      auto issue_pv = [&](int mt, int stage, bool accumulate) {
-        const uint32_t vb = ring_addr + stage * C::kStageBytes;
-#pragma unroll
-        for (int kk = 0; kk < SPX_TILE_KEYS / 16; ++kk)
-          mma_ts(tmem + mt * 128, tmem + 256 + mt * 128 + kk * 8,
-                 smem_desc_sw128(vb + kk * 2048, kSubTileBytes, 1024), idesc_o, (accumulate || kk > 0) ? 1u : 0u);
-      };
+      }
+      ctl->anc[t] = m;
+    }
+    tc_fence_before();
+    named_bar_sync(1, kThreads - 32);
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
 
-      for (int u = unit_lo; u < unit_hi && ok;) {
-        const int prob = u / p.UPP;
-        const int tile_lo = u - prob * p.UPP;
-        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
-        const int n = tile_hi - tile_lo;
-        ok = mbar_wait(&ctl->q_full, seg & 1, abort_flag);
-        if (!ok) break;
-        {
-          const int ks = kvc % NS;
-          ok = mbar_wait(&ctl->kv_full[ks], (kvc / NS) & 1, abort_flag);
+    if (warp == kMmaWarp) {
+      // ================================ MMA issuer ==========================================
+      setmaxnreg_dec<kRegsOther>();
+      if (lane == 0) {
+        const uint32_t idesc_s = idesc_bf16_f32(128, SPX_TILE_KEYS, false, false);
+        const uint32_t idesc_o = idesc_bf16_f32(128, D, false, true);
+        constexpr uint32_t hi = desc_hi(1024);
+        const uint32_t q_lo = desc_lo(smem_u32(Qs), 16);
+        const uint32_t k_lo0 = desc_lo(smem_u32(ring), 16);
+        const uint32_t v_lo0 = desc_lo(smem_u32(ring), kSubTileBytes);
+        uint32_t kvc = 0, it = 0;
+        int seg = 0;
+
+        auto issue_s = [&](int mt, int stage) {
+          const uint32_t kb = k_lo0 + stage * (C::kStageBytes >> 4);
+          const uint32_t qb = q_lo + mt * (DS * kSubTileBytes >> 4);
+          const uint32_t d = tmem + 256 + mt * 128;
+#pragma unroll
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * (kSubTileBytes >> 4) + (kk & 3) * 2;
+            mma_ss2(d, qb + off, hi, kb + off, hi, idesc_s, kk > 0 ? 1u : 0u);
+          }
+          mma_commit(&ctl->s_full[mt]);
+        };
+        auto issue_pv = [&](int mt, int stage, uint32_t accumulate) {
+          const uint32_t vb = v_lo0 + stage * (C::kStageBytes >> 4);
+          const uint32_t d = tmem + mt * 128;
+          const uint32_t pa = tmem + 256 + mt * 128;
+          mma_ts2(d, pa, vb, hi, idesc_o, accumulate);
+#pragma unroll
+          for (int kk = 1; kk < SPX_TILE_KEYS / 16; ++kk) mma_ts2(d, pa + kk * 8, vb + kk * 128, hi, idesc_o, 1u);
+        };
+
+        for (int u = unit_lo; u < unit_hi && ok;) {
+          const int prob = u / p.UPP;
+          const int tile_lo = u - prob * p.UPP;
+          const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+          const int n = tile_hi - tile_lo;
+          ok = mbar_wait(&ctl->q_full, seg & 1, abort_flag);
           if (!ok) break;
-          tc_fence_after();
-          for (int mt = 0; mt < n_mt; ++mt) issue_s(mt, ks);
-          mma_commit(&ctl->kv_empty[ks]);
-          ++kvc;
-        }
-        for (int i = 0; i < n && ok; ++i) {
-          const bool has_next = i + 1 < n, last = !has_next;
-          const int vs = kvc % NS;
-          const uint32_t vph = (kvc / NS) & 1;
-          ++kvc;
-          const int ks = kvc % NS;
-          const uint32_t kph = (kvc / NS) & 1;
-          ok = mbar_wait(&ctl->kv_full[vs], vph, abort_flag);
-          for (int mt = 0; mt < n_mt && ok; ++mt) {
-            ok = mbar_wait(&ctl->p_full[mt], it & 1, abort_flag);
-            if (ok && i == 0 && seg > 0) ok = mbar_wait(&ctl->o_free[mt], (seg - 1) & 1, abort_flag);
+          {
+            const int ks = kvc % NS;
+            ok = mbar_wait(&ctl->kv_full[ks], (kvc / NS) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            issue_pv(mt, vs, i > 0);
-            if (last) mma_commit(&ctl->o_done[mt]);
-            if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[vs]);
-            if (has_next) {
-              if (mt == 0) {
-                ok = mbar_wait(&ctl->kv_full[ks], kph, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
+            SPX_EVT(1, 0);
+            for (int mt = 0; mt < n_mt; ++mt) issue_s(mt, ks);
+            mma_commit(&ctl->kv_empty[ks]);
+            SPX_EVT(1, 1);
+            ++kvc;
+          }
+          for (int i = 0; i < n && ok; ++i) {
+            const bool has_next = i + 1 < n, last = !has_next;
+            const int vs = kvc % NS;
+            const uint32_t vph = (kvc / NS) & 1;
+            ++kvc;
+            const int ks = kvc % NS;
+            const uint32_t kph = (kvc / NS) & 1;
+            ok = mbar_wait(&ctl->kv_full[vs], vph, abort_flag);
+            for (int mt = 0; mt < n_mt && ok; ++mt) {
+              SPX_EVT(2, it * 4 + mt * 2);
+              ok = mbar_wait(&ctl->p_full[mt], it & 1, abort_flag);
+              SPX_EVT(2, it * 4 + mt * 2 + 1);
+              if (ok && i == 0 && seg > 0) ok = mbar_wait(&ctl->o_free[mt], (seg - 1) & 1, abort_flag);
+              if (!ok) break;
+              tc_fence_after();
+              SPX_EVT(1, 2 + it * 4 + mt * 2);
+              issue_pv(mt, vs, i > 0 ? 1u : 0u);
+              if (last) mma_commit(&ctl->o_done[mt]);
+              if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[vs]);
+              if (has_next) {
+                if (mt == 0) {
+                  ok = mbar_wait(&ctl->kv_full[ks], kph, abort_flag);
+                  if (!ok) break;
+                  tc_fence_after();
+                }
+                issue_s(mt, ks);
+                if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[ks]);
               }
-              issue_s(mt, ks);
-              if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[ks]);
+              SPX_EVT(1, 3 + it * 4 + mt * 2);
             }
+            if (has_next) ++kvc;
+            ++it;
           }
-          if (has_next) ++kvc;
-          ++it;
+          if (ok) mma_commit(&ctl->q_free);
+          u += n;
+          ++seg;
         }
-        if (ok) mma_commit(&ctl->q_free);
-        u += n;
-        ++seg;
+        // drain: all MMAs issued so far must have completed before tensor memory is released
+        mma_commit(&ctl->drain);
+        for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(&ctl->drain, 0); ++spin) {}
       }
-      // drain: all MMAs issued so far must have completed before tensor memory is released
-      mma_commit(&ctl->drain);
-      for (int spin = 0; spin < (1 << 22) && !mbar_try_wait(&ctl->drain, 0); ++spin) {}
-    }
-  } else {
-    // ================================ softmax warps =========================================
-    const int mt = (warp - 2) >> 2;
-    if (mt < n_mt) {
-      const int quarter = warp & 3;
-      const int row_t = quarter * 32 + lane;
-      const int rr = mt * 128 + row_t;
-      const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-      const uint32_t s_addr = tmem + lane_addr + 256 + mt * 128;
-      const uint32_t o_addr = tmem + lane_addr + mt * 128;
-      const float scale2 = p.scale2;
-      uint32_t it = 0;
-      int seg = 0;
-      for (int u = unit_lo; u < unit_hi && ok;) {
-        const int prob = u / p.UPP;
-        const int tile_lo = u - prob * p.UPP;
-        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
-        const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
-        const int r = rblk * p.RB + rr;
-        const bool valid = r < p.rows;
-        const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
-        float m_used = -INFINITY, l = 0.f;
+    } else if (warp > kMmaWarp) {
+      setmaxnreg_dec<kRegsOther>();
+    } else {
+      // ================================ softmax warps =======================================
+      setmaxnreg_inc<kRegsSoftmax>();
+      const int mt = warp >> 2;
+      if (mt < n_mt) {
+        const int quarter = warp & 3;
+        const int row_t = quarter * 32 + lane;
+        const int rr = mt * 128 + row_t;
+        const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+        const uint32_t s_addr = tmem + lane_addr + 256 + mt * 128;
+        const uint32_t o_addr = tmem + lane_addr + mt * 128;
+        const float scale2 = p.scale2;
+        uint32_t it = 0;
+        int seg = 0;
+        for (int u = unit_lo; u < unit_hi && ok;) {
+          const int prob = u / p.UPP;
+          const int tile_lo = u - prob * p.UPP;
+          const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+          const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+          const int r = rblk * p.RB + rr;
+          const bool valid = r < p.rows;
+          const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
+          float m_used = -INFINITY, l = 0.f;
 
-        for (int tile = tile_lo; tile < tile_hi; ++tile, ++it) {
-          const bool is_tree = tile == p.TPH;
-          const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
-          const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
-          unsigned long long vis_lo = ~0ull, vis_hi = ~0ull;
-          if (is_tree) {
-            vis_lo = tree_mask;
-            vis_hi = 0ull;
-          } else if (need_mask) {
-            vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
-            vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);
-          }
-          ok = mbar_wait(&ctl->s_full[mt], it & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
+          for (int tile = tile_lo; tile < tile_hi; ++tile, ++it) {
+            const bool is_tree = tile == p.TPH;
+            const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
+            const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
+            ok = mbar_wait(&ctl->s_full[mt], it & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) SPX_EVT(4 + warp, it * 4);
 
-          // pass 1: maximum of the visible raw scores of this row
-          float tmax = -INFINITY;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t v[32];
-            tmem_ld32(s_addr + c * 32, v);
+            // the whole S row of this thread: 128 fp32 scores in registers
+            uint32_t s0[32], s1[32], s2[32], s3[32];
+            tmem_ld32(s_addr, s0);
+            tmem_ld32(s_addr + 32, s1);
+            tmem_ld32(s_addr + 64, s2);
+            tmem_ld32(s_addr + 96, s3);
             tmem_wait_ld();
             if (need_mask) {
-              const uint32_t bits = static_cast<uint32_t>((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32));
+              unsigned long long vis_lo, vis_hi;
+              if (is_tree) {
+                vis_lo = tree_mask;
+                vis_hi = 0ull;
+              } else {
+                vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
+                vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);
+              }
+              const uint32_t b0 = static_cast<uint32_t>(vis_lo), b1 = static_cast<uint32_t>(vis_lo >> 32);
+              const uint32_t b2 = static_cast<uint32_t>(vis_hi), b3 = static_cast<uint32_t>(vis_hi >> 32);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (!((b0 >> j) & 1u)) s0[j] = 0xff800000u;    // -inf
+                if (!((b1 >> j) & 1u)) s1[j] = 0xff800000u;
+                if (!((b2 >> j) & 1u)) s2[j] = 0xff800000u;
+                if (!((b3 >> j) & 1u)) s3[j] = 0xff800000u;
+              }
+            }
+            float t0 = -INFINITY, t1 = -INFINITY, t2 = -INFINITY, t3 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              t0 = fmax3(t0, __uint_as_float(s0[j]), __uint_as_float(s0[j + 1]));
+              t1 = fmax3(t1, __uint_as_float(s1[j]), __uint_as_float(s1[j + 1]));
+              t2 = fmax3(t2, __uint_as_float(s2[j]), __uint_as_float(s2[j + 1]));
+              t3 = fmax3(t3, __uint_as_float(s3[j]), __uint_as_float(s3[j + 1]));
+            }
+            const float tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 1);
+            const float m_tile = tmax * scale2;
+            float alpha = 1.f;
+            bool rescale = false;
+            if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
+              alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
+              rescale = tile > tile_lo;
+              m_used = m_tile;
+              l *= alpha;
+            }
+            if (__any_sync(0xffffffffu, rescale)) {
+              // S(tile) has been committed after PV(tile-1), so O is complete and not being written
+#pragma unroll
+              for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(o_addr + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
+                tmem_st32(o_addr + c * 32, v);
+              }
+            }
+
+            // exponentials against the reference maximum, sums, P in bf16 back to tensor memory
+            const float neg_m = -m_used;
+            const bool score = SCORE && !is_tree;
+            float* mass = nullptr;
+            if (score) {
+              const long long rowbase = ((long long)prob * p.TPH + tile) * p.RB + rr;
+              mass = a.ws + p.off_mass + rowbase * p.CPT;
+              a.ws[p.off_mref + rowbase] = m_used;
+            }
+            float csum = 0.f;
+            auto exp_chunk = [&](uint32_t (&v)[32], int c) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                tmax = fmaxf(tmax, ((bits >> j) & 1u) ? __uint_as_float(v[j]) : -INFINITY);
-            } else {
+                v[j] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(v[j]), scale2, neg_m)));
+              float gs0 = 0.f, gs1 = 0.f, gs2 = 0.f, gs3 = 0.f;
 #pragma unroll
-              for (int j = 0; j < 32; ++j) tmax = fmaxf(tmax, __uint_as_float(v[j]));
-            }
+              for (int j = 0; j < 32; j += 4) {
+                gs0 += __uint_as_float(v[j]);
+                gs1 += __uint_as_float(v[j + 1]);
+                gs2 += __uint_as_float(v[j + 2]);
+                gs3 += __uint_as_float(v[j + 3]);
+              }
+              const float gs = (gs0 + gs1) + (gs2 + gs3);
+              l += gs;
+              if (score) {
+                if (p.C >= 32) {
+                  csum += gs;
+                  if ((((c + 1) * 32) & (p.C - 1)) == 0) {
+                    mass[((c + 1) * 32) / p.C - 1] = csum;
+                    csum = 0.f;
+                  }
+                } else {
+                  float acc = 0.f;
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) {
+                    acc += __uint_as_float(v[j]);
+                    if (((j + 1) & (p.C - 1)) == 0) {
+                      mass[(c * 32 + j) / p.C] = acc;
+                      acc = 0.f;
+                    }
+                  }
+                }
+              }
+              uint32_t pk[16];
+#pragma unroll
+              for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              tmem_st16(s_addr + c * 16, pk);
+            };
+            exp_chunk(s0, 0);
+            exp_chunk(s1, 1);
+            exp_chunk(s2, 2);
+            exp_chunk(s3, 3);
+            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 2);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&ctl->p_full[mt]);
+            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 3);
           }
-          const float m_tile = tmax * scale2;
-          float alpha = 1.f;
-          bool rescale = false;
-          if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
-            alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
-            rescale = tile > tile_lo;
-            m_used = m_tile;
-            l *= alpha;
-          }
-          if (__any_sync(0xffffffffu, rescale)) {
-            // S(tile) has been committed after PV(tile-1), so O is complete and not being written
+          if (!ok) break;
+
+          // epilogue of the segment: unnormalised O, reference maximum and row sum to the partial slot
+          ok = mbar_wait(&ctl->o_done[mt], seg & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) SPX_EVT(4 + warp, 60 + (seg & 1) * 2);
+          {
+            const int slot = cta + prob;
+            float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
               uint32_t v[32];
               tmem_ld32(o_addr + c * 32, v);
               tmem_wait_ld();
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * alpha);
-              tmem_st32(o_addr + c * 32, v);
-            }
-          }
-
-          // pass 2: exponentials against the reference maximum, sums, P in bf16 back to tensor memory
-          const float neg_m = -m_used;
-          const bool score = SCORE && !is_tree;
-          float* mass = nullptr;
-          if (score) {
-            const long long rowbase = ((long long)prob * p.TPH + tile) * p.RB + rr;
-            mass = a.ws + p.off_mass + rowbase * p.CPT;
-            a.ws[p.off_mref + rowbase] = m_used;
-          }
-          float csum = 0.f;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t v[32];
-            tmem_ld32(s_addr + c * 32, v);
-            tmem_wait_ld();
-            const uint32_t bits = need_mask ? static_cast<uint32_t>((c < 2 ? vis_lo : vis_hi) >> ((c & 1) * 32))
-                                            : 0xffffffffu;
-            float pr[32];
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              float x = fmaf(__uint_as_float(v[j]), scale2, neg_m);
-              if (need_mask) x = ((bits >> j) & 1u) ? x : -INFINITY;
-              pr[j] = ex2_approx(x);
-            }
-            float gs0 = 0.f, gs1 = 0.f, gs2 = 0.f, gs3 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              gs0 += pr[j];
-              gs1 += pr[j + 1];
-              gs2 += pr[j + 2];
-              gs3 += pr[j + 3];
-            }
-            const float gs = (gs0 + gs1) + (gs2 + gs3);
-            l += gs;
-            if (score) {
-              if (p.C >= 32) {
-                csum += gs;
-                if ((((c + 1) * 32) & (p.C - 1)) == 0) {
-                  mass[((c + 1) * 32) / p.C - 1] = csum;
-                  csum = 0.f;
-                }
-              } else {
-                float acc = 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                  acc += pr[j];
-                  if (((j + 1) & (p.C - 1)) == 0) {
-                    mass[(c * 32 + j) / p.C] = acc;
-                    acc = 0.f;
-                  }
-                }
+              for (int q4 = 0; q4 < 8; ++q4) {
+                const float4 x = make_float4(__uint_as_float(v[q4 * 4]), __uint_as_float(v[q4 * 4 + 1]),
+                                             __uint_as_float(v[q4 * 4 + 2]), __uint_as_float(v[q4 * 4 + 3]));
+                *reinterpret_cast<float4*>(po + ((long long)(c * 8 + q4) * p.RB + rr) * 4) = x;
               }
             }
-            uint32_t pk[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(pr[2 * j], pr[2 * j + 1]);
-            tmem_st16(s_addr + c * 16, pk);
+            a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_used;
+            a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l;
           }
-          tmem_wait_st();
+          if (lane == 0) SPX_EVT(4 + warp, 61 + (seg & 1) * 2);
           tc_fence_before();
-          mbar_arrive(&ctl->p_full[mt]);
+          mbar_arrive(&ctl->o_free[mt]);
+          u += tile_hi - tile_lo;
+          ++seg;
         }
-        if (!ok) break;
-
-        // epilogue of the segment: unnormalised O, reference maximum and row sum to the partial slot
-        ok = mbar_wait(&ctl->o_done[mt], seg & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        {
-          const int slot = cta + prob;
-          float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(o_addr + c * 32, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              const float4 x = make_float4(__uint_as_float(v[q4 * 4]), __uint_as_float(v[q4 * 4 + 1]),
-                                           __uint_as_float(v[q4 * 4 + 2]), __uint_as_float(v[q4 * 4 + 3]));
-              *reinterpret_cast<float4*>(po + ((long long)(c * 8 + q4) * p.RB + rr) * 4) = x;
-            }
-          }
-          a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_used;
-          a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l;
-        }
-        tc_fence_before();
-        mbar_arrive(&ctl->o_free[mt]);
-        u += tile_hi - tile_lo;
-        ++seg;
       }
     }
   }
@@ -405,9 +469,10 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
   if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (tid == 0) SPX_EVT(0, 63);
+  if (warp == kMmaWarp) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(ctl->tmem_base, 512);
   }
 }
 

@@ -23,7 +23,20 @@ struct AttnArgs {
   float* ws;
   int32_t* status;
   long long q_st, q_sh, kv_sl, kv_sh, tkv_st, tkv_sh, o_st, o_sh;
+#ifdef SPX_TRACE
+  long long* trace;   // timing trace of two CTAs (development builds only)
+#endif
 };
+
+#ifdef SPX_TRACE
+#define SPX_EVT(role, idx)                                                                              \
+  do {                                                                                                  \
+    if (a.trace && (blockIdx.x == 0 || blockIdx.x == 77) && (idx) < 64)                                 \
+      a.trace[((blockIdx.x ? 1 : 0) * 12 + (role)) * 64 + (idx)] = clock64() - spx_t_start;              \
+  } while (0)
+#else
+#define SPX_EVT(role, idx) do {} while (0)
+#endif
 
 __device__ __forceinline__ void spx_raise(int32_t* status, int code) {
   if (status) atomicOr(status, 1 << code);

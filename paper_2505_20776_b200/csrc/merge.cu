@@ -1,8 +1,7 @@
 // Log-sum-exp merge of the per-segment partial results, and the normalisation of the per-chunk
 // sums into the head-averaged chunk scores that retrieval ranks.
 //
-// merge_kernel: one CTA = 32 query rows of one problem (warp = one 16-byte column group over the
-// 32 rows, so partial reads are 512-byte coalesced).  For each row: M = max_s m_s,
+// merge_kernel: for each query row: M = max_s m_s,
 // Z = sum_s l_s 2^(m_s - M), lse = (M + log2 Z) ln 2, O = sum_s O~_s 2^(m_s - M) / Z.
 //
 // score_kernel: one thread per (tree node, chunk): sums over all query heads the chunk's
@@ -15,67 +14,74 @@ namespace {
 constexpr float kLn2 = 0.693147180559945309417f;
 constexpr float kLog2e = 1.44269504088896340736f;
 
-__global__ void __launch_bounds__(128) merge_kernel(const __grid_constant__ AttnArgs a) {
+// Block = 8 warps; warp w handles one 16-byte column group d4 for 32 consecutive rows of one
+// problem, so every partial read is a 512-byte coalesced segment and all reads of a thread are
+// independent of each other.
+__global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
-  extern __shared__ float wsm[];                       // [max_segs][32] merge weights
   const int blocks_per_prob = p.RB / 32;
   const int prob = blockIdx.x / blocks_per_prob;
   const int rr0 = (blockIdx.x - prob * blocks_per_prob) * 32;
   const int g = prob / p.n_rblk;
   const int rblk = prob - g * p.n_rblk;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int rr = rr0 + lane;
+  const int r = rblk * p.RB + rr;
+  if (r >= p.rows) return;
   const int c_first = spx_unit_owner(p, prob * p.UPP);
   const int c_last = spx_unit_owner(p, (prob + 1) * p.UPP - 1);
   const int nseg = c_last - c_first + 1;
   const int slot0 = c_first + prob;
-  if (rblk * p.RB + rr0 >= p.rows) return;             // whole CTA beyond the valid rows
-
-  const int rr = rr0 + lane;
-  const int r = rblk * p.RB + rr;
-  const bool valid = r < p.rows;
-  if (warp == 0) {
-    float M = -INFINITY;
-    for (int s = 0; s < nseg; ++s) M = fmaxf(M, a.ws[p.off_part_m + (long long)(slot0 + s) * p.RB + rr]);
-    float Z = 0.f;
-    for (int s = 0; s < nseg; ++s) {
-      const float ms = a.ws[p.off_part_m + (long long)(slot0 + s) * p.RB + rr];
-      const float ls = a.ws[p.off_part_l + (long long)(slot0 + s) * p.RB + rr];
-      const float w = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
-      Z += ls * w;
-      wsm[s * 32 + lane] = w;
-    }
-    const float inv = 1.f / Z;
-    for (int s = 0; s < nseg; ++s) wsm[s * 32 + lane] *= inv;
-    if (valid && blockIdx.y == 0) {
-      const int t = r / p.G, h = g * p.G + r % p.G;
-      a.lse[(long long)h * p.T + t] = (M + log2f(Z)) * kLn2;
-    }
-  }
-  __syncthreads();
-  if (!valid) return;
-
   const int nd4 = p.D / 4;
-  const int per_y = nd4 / gridDim.y;
-  const int t = r / p.G, h = g * p.G + r % p.G;
-  __nv_bfloat16* orow = a.O + (long long)t * a.o_st + (long long)h * a.o_sh;
-  for (int d4 = blockIdx.y * per_y + warp; d4 < (blockIdx.y + 1) * per_y; d4 += 4) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < nseg; ++s) {
-      const float w = wsm[s * 32 + lane];
-      const float4 v = *reinterpret_cast<const float4*>(
-          a.ws + p.off_part_o + (((long long)(slot0 + s) * nd4 + d4) * p.RB + rr) * 4);
-      acc.x = fmaf(w, v.x, acc.x);
-      acc.y = fmaf(w, v.y, acc.y);
-      acc.z = fmaf(w, v.z, acc.z);
-      acc.w = fmaf(w, v.w, acc.w);
+  const int d4 = blockIdx.y * 8 + warp;
+
+  const float* pm = a.ws + p.off_part_m + (long long)slot0 * p.RB + rr;
+  const float* pl = a.ws + p.off_part_l + (long long)slot0 * p.RB + rr;
+  const float* po = a.ws + p.off_part_o + (((long long)slot0 * nd4 + d4) * p.RB + rr) * 4;
+  const long long ostride = (long long)nd4 * p.RB * 4;
+
+  float M = -INFINITY;
+  for (int s = 0; s < nseg; ++s) M = fmaxf(M, pm[(long long)s * p.RB]);
+  float Z = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  int s = 0;
+  for (; s + 4 <= nseg; s += 4) {
+    float ms[4], ls[4];
+    float4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      ms[k] = pm[(long long)(s + k) * p.RB];
+      ls[k] = pl[(long long)(s + k) * p.RB];
+      v[k] = *reinterpret_cast<const float4*>(po + (s + k) * ostride);
     }
-    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(orow + d4 * 4) = pk;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float w = exp2f(ms[k] - M);
+      Z = fmaf(ls[k], w, Z);
+      acc.x = fmaf(w, v[k].x, acc.x);
+      acc.y = fmaf(w, v[k].y, acc.y);
+      acc.z = fmaf(w, v[k].z, acc.z);
+      acc.w = fmaf(w, v[k].w, acc.w);
+    }
   }
+  for (; s < nseg; ++s) {
+    const float w = exp2f(pm[(long long)s * p.RB] - M);
+    const float4 v = *reinterpret_cast<const float4*>(po + s * ostride);
+    Z = fmaf(pl[(long long)s * p.RB], w, Z);
+    acc.x = fmaf(w, v.x, acc.x);
+    acc.y = fmaf(w, v.y, acc.y);
+    acc.z = fmaf(w, v.z, acc.z);
+    acc.w = fmaf(w, v.w, acc.w);
+  }
+  const float inv = 1.f / Z;
+  const int t = r / p.G, h = g * p.G + r % p.G;
+  if (d4 == 0) a.lse[(long long)h * p.T + t] = (M + log2f(Z)) * kLn2;
+  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+  __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  uint2 pk;
+  pk.x = *reinterpret_cast<uint32_t*>(&lo);
+  pk.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
 }
 
 __global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ AttnArgs a) {
@@ -102,9 +108,8 @@ __global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ Attn
 
 cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches) {
   const AttnPlan& p = a.plan;
-  const int ysplit = (p.D / 4) % 8 == 0 ? 2 : 1;
-  const dim3 grid(p.NP * (p.RB / 32), ysplit);
-  merge_kernel<<<grid, 128, (size_t)p.max_segs * 32 * sizeof(float), st>>>(a);
+  const dim3 grid(p.NP * (p.RB / 32), p.D / 32);
+  merge_kernel<<<grid, 256, 0, st>>>(a);
   *n_launches += 1;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -358,3 +358,38 @@ def test_determinism_run_to_run(cuda_device):
     for o in outs[1:]:
         for a, b in zip(o, outs[0]):
             assert torch.equal(a, b)
+
+
+def test_tensor_core_kernel_agrees_with_cuda_core_kernel(cuda_device):
+    """Two independent device implementations of the split attention must agree closely."""
+    w = synth.WORKLOADS["c1"]
+    dev = cuda_device
+    t = to_dev(synth.make_layer(w), dev)
+    par = torch.from_numpy(synth.make_tree(w)).to(dev)
+    outs = []
+    try:
+        for kernel in (1, 2):
+            api.specext_set_tuning(kernel, 0)
+            hp = make_hp(w, dev)
+            hp.verify_attn(t, par, w.prefix_len, True)
+            assert hp.read_status() == 0
+            outs.append((hp.O.float().clone(), hp.lse.clone(), hp.chunk_score(w.prefix_len).clone()))
+    finally:
+        api.specext_set_tuning(0, 0)
+    assert (outs[0][0] - outs[1][0]).abs().max().item() <= 2e-2
+    assert (outs[0][1] - outs[1][1]).abs().max().item() <= 1e-4
+    rel = ((outs[0][2] - outs[1][2]).abs() / outs[0][2]).max().item()
+    assert rel <= 1e-4
+
+
+def test_coarser_splits_give_the_same_result(cuda_device):
+    w = synth.WORKLOADS["c1"]
+    dev = cuda_device
+    t_cpu = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    try:
+        api.specext_set_tuning(0, 5)
+        hp = make_hp(w, dev)
+        check_attn(hp, t_cpu, parent, w.prefix_len, w.chunk_size)
+    finally:
+        api.specext_set_tuning(0, 1)
