@@ -150,6 +150,35 @@ const char* specext_status_string(int status);
 int64_t specext_launch_count(void);
 
 /*
+ * specext_verify_attn for callers that cannot allocate device memory (the paper has no counterpart).
+ *
+ * Some callers have nowhere to get the scratch buffer from: code that runs after the process has
+ * handed all device memory to a pool it does not own, plug-ins that are forbidden to call
+ * cudaMalloc, or a recovery path that must keep working when the allocator has failed.  This entry
+ * point takes the same inputs and outputs as specext_verify_attn but no workspace: the scratch is a
+ * fixed array of SPECEXT_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU
+ * that loads the library holds that much memory until the process exits.
+ *
+ *   - Shapes whose scratch need (specext_verify_attn_workspace) exceeds
+ *     SPECEXT_STATIC_SCRATCH_BYTES are rejected with SPECEXT_ERR_WORKSPACE; nothing is launched.
+ *   - The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current) and caches it; make that first call outside of any stream capture.
+ *   - All calls on a device share the one array.  Calls must therefore not overlap on the GPU:
+ *     order them on one stream (or by events); two calls running concurrently race on the scratch
+ *     and both produce garbage.  Nothing in the array has to survive from one call to the next and
+ *     nothing has to start at zero: every call rewrites the part it reads.
+ * Arguments, outputs, arithmetic and error reporting are those of specext_verify_attn.
+ */
+#define SPECEXT_STATIC_SCRATCH_BYTES (32u << 20)
+int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void* Q,
+                                       const void* K_prefix, const void* V_prefix,
+                                       const void* K_tree, const void* V_tree,
+                                       const int32_t* parent, void* O, float* lse,
+                                       float* chunk_score, int32_t* device_status,
+                                       void* cuda_stream);
+
+/*
  * Process-wide tuning and cross-check switches (the paper has no counterpart).
  *   attn_kernel       : 0 or 2 = tensor-core (tcgen05) attention kernel, the default;
  *                       1 = the CUDA-core kernel, an independent on-device cross-check.

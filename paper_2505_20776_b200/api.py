@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
     L.specext_verify_attn_workspace.argtypes = [ctypes.POINTER(AttnDesc)]
     L.specext_verify_attn.restype = ctypes.c_int
     L.specext_verify_attn.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9 + [vp, sz, vp, vp]
+    L.specext_verify_attn_static_scratch.restype = ctypes.c_int
+    L.specext_verify_attn_static_scratch.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9 + [vp, vp]
     L.specext_select_chunks.restype = ctypes.c_int
     L.specext_select_chunks.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     L.specext_gather_kv.restype = ctypes.c_int
@@ -135,6 +137,27 @@ def specext_verify_attn(desc: AttnDesc, Q: torch.Tensor, K_prefix: torch.Tensor,
                                    _ptr(workspace), workspace.numel() * workspace.element_size(),
                                    _ptr(device_status), _stream())
     _check(rc, "specext_verify_attn")
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def specext_verify_attn_static_scratch(desc: AttnDesc, Q: torch.Tensor, K_prefix: torch.Tensor,
+                                       V_prefix: torch.Tensor, K_tree: torch.Tensor, V_tree: torch.Tensor,
+                                       parent: torch.Tensor, O: torch.Tensor, lse: torch.Tensor,
+                                       chunk_score: Optional[torch.Tensor], device_status: torch.Tensor) -> None:
+    """specext_verify_attn without a workspace argument: for callers that may not allocate device memory.
+
+    The scratch is a fixed 32 MiB array inside the library; shapes that need more raise
+    SPECEXT_ERR_WORKSPACE.  Calls on one device share that array and must not overlap on the GPU.
+    The first call on a device should be made outside of stream capture.
+    """
+    if V_prefix.stride() != K_prefix.stride() or V_tree.stride() != K_tree.stride():
+        raise ValueError("V tensors must have the strides of the matching K tensors")
+    rc = lib().specext_verify_attn_static_scratch(ctypes.byref(desc), _ptr(Q), _ptr(K_prefix), _ptr(V_prefix),
+                                                  _ptr(K_tree), _ptr(V_tree), _ptr(parent), _ptr(O), _ptr(lse),
+                                                  _ptr(chunk_score), _ptr(device_status), _stream())
+    _check(rc, "specext_verify_attn_static_scratch")
 
 
 def specext_select_chunks(chunk_score: torch.Tensor, row: int, prefix_len: int, chunk_size: int, k: int,

@@ -12,7 +12,15 @@ cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int 
                               const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
                               int32_t* n_tokens_out, int32_t* status, cudaStream_t st);
 
+// Scratch of the entry point that takes no workspace.  Part of the library image: resident on every
+// device that loads the library until the process exits.  Device code may name it directly; host
+// code must go through cudaGetSymbolAddress (see specext_verify_attn_static_scratch).
+static __device__ __align__(256) unsigned char g_static_scratch[SPECEXT_STATIC_SCRATCH_BYTES];
+
 namespace {
+
+constexpr int kMaxDevices = 64;
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_attn_kernel{0};       // 0 = default, 1 = CUDA-core kernel, 2 = tensor-core kernel
@@ -151,6 +159,36 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
     return SPECEXT_ERR_CUDA;
   }
   return SPECEXT_OK;
+}
+
+int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void* Q,
+                                       const void* K_prefix, const void* V_prefix,
+                                       const void* K_tree, const void* V_tree,
+                                       const int32_t* parent, void* O, float* lse,
+                                       float* chunk_score, int32_t* device_status,
+                                       void* cuda_stream) {
+  // Reject a bad descriptor, or a shape that does not fit, before touching the device.
+  AttnPlan plan;
+  const int rc = build_plan(desc, &plan);
+  if (rc != SPECEXT_OK) return rc;
+  if ((size_t)plan.total_floats * sizeof(float) > SPECEXT_STATIC_SCRATCH_BYTES) return SPECEXT_ERR_WORKSPACE;
+  // g_static_scratch names a host-side handle of the device array, not a device address: the address
+  // valid on the current device comes from cudaGetSymbolAddress, looked up once per device.
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return SPECEXT_ERR_CUDA;
+  }
+  void* scratch = g_static_scratch_addr[dev].load();
+  if (!scratch) {
+    if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || !scratch) {
+      (void)cudaGetLastError();
+      return SPECEXT_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev].store(scratch);
+  }
+  return specext_verify_attn(desc, Q, K_prefix, V_prefix, K_tree, V_tree, parent, O, lse, chunk_score, scratch,
+                             SPECEXT_STATIC_SCRATCH_BYTES, device_status, cuda_stream);
 }
 
 int specext_select_chunks(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
