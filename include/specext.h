@@ -180,7 +180,10 @@ int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void
 
 /*
  * Process-wide tuning and cross-check switches (the paper has no counterpart).
- *   attn_kernel       : 0 or 2 = tensor-core (tcgen05) attention kernel, the default;
+ *   attn_kernel       : 0 = default: the paired-CTA tensor-core (tcgen05 cta_group::2) kernel for
+ *                       head_dim 128 with more than 128 stacked query rows per KV head, else the
+ *                       one-CTA tensor-core kernel; 2 / 3 = force the one-CTA / paired kernel
+ *                       (3 falls back to 2 for shapes the paired kernel is not built for);
  *                       1 = the CUDA-core kernel, an independent on-device cross-check.
  *   min_tiles_per_cta : lower bound on the 128-key tiles one CTA processes (> 0 to change; fewer,
  *                       longer splits mean fewer partial results to merge).  Changes the

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libspecext.so")
-SOURCES = ["api.cu", "attn_tc.cu", "attn_simt.cu", "merge.cu", "retrieval.cu"]
+SOURCES = ["api.cu", "attn_tc2.cu", "attn_tc.cu", "attn_simt.cu", "merge.cu", "retrieval.cu"]
 
 
 def nvcc_path() -> str:

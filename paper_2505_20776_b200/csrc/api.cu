@@ -75,15 +75,40 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   if (U > (1ll << 30)) return SPECEXT_ERR_UNSUPPORTED;
   p.U = (int)U;
   const int min_units = g_min_units.load() < 1 ? 1 : g_min_units.load();
-  int n_cta = p.U / min_units;
-  if (n_cta < 1) n_cta = 1;
-  if (n_cta > sm_count()) n_cta = sm_count();
-  p.n_cta = n_cta;
-  p.q = p.U / n_cta;
-  p.rem = p.U % n_cta;
-  p.n_slots = n_cta + p.NP - 1;
-  p.max_segs = (p.UPP + p.q - 1) / p.q + 1;
-  if (p.max_segs > n_cta) p.max_segs = n_cta;
+  const int want = g_attn_kernel.load();
+  const bool pair_ok = p.D == 128 && p.RB == 256;       // what the paired-CTA kernel is built for
+  p.kernel = want == 1 ? 1 : ((want == 0 || want == 3) && pair_ok ? 3 : 2);
+  if (p.kernel == 3) {
+    // one worker = a cluster of two CTAs; every problem gets the same number of workers when possible
+    const int n_workers = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+    if (p.NP <= n_workers) {
+      int cpp = n_workers / p.NP;
+      if (cpp > p.UPP / min_units) cpp = p.UPP / min_units;
+      if (cpp < 1) cpp = 1;
+      p.cpp = cpp;
+      p.n_cta = p.NP * cpp;
+      p.q = p.UPP / cpp;
+      p.rem = p.UPP % cpp;
+      p.max_segs = cpp;
+    } else {
+      p.cpp = 0;
+      p.n_cta = n_workers;
+      p.q = p.U / p.n_cta;
+      p.rem = p.U % p.n_cta;
+      p.max_segs = (p.UPP + p.q - 1) / p.q + 1;
+    }
+  } else {
+    int n_cta = p.U / min_units;
+    if (n_cta < 1) n_cta = 1;
+    if (n_cta > sm_count()) n_cta = sm_count();
+    p.cpp = 0;
+    p.n_cta = n_cta;
+    p.q = p.U / n_cta;
+    p.rem = p.U % n_cta;
+    p.max_segs = (p.UPP + p.q - 1) / p.q + 1;
+  }
+  if (p.max_segs > p.n_cta) p.max_segs = p.n_cta;
+  p.n_slots = p.n_cta + p.NP - 1;
   p.CPT = SPX_TILE_KEYS / p.C;
   p.NC = (p.L + p.C - 1) / p.C;
   p.want_score = d->want_chunk_score != 0;
@@ -151,7 +176,9 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int n = 0;
-  cudaError_t e = g_attn_kernel.load() == 1 ? spx_launch_attn_simt(a, st, &n) : spx_launch_attn_tc(a, st, &n);
+  cudaError_t e = p.kernel == 1   ? spx_launch_attn_simt(a, st, &n)
+                  : p.kernel == 3 ? spx_launch_attn_tc2(a, st, &n)
+                                  : spx_launch_attn_tc(a, st, &n);
   if (e == cudaSuccess) e = spx_launch_merge(a, st, &n);
   g_launches.fetch_add(n);
   if (e != cudaSuccess) {
@@ -278,7 +305,7 @@ void specext_debug_set_trace(void* p) { g_trace = static_cast<long long*>(p); }
 #endif
 
 int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta) {
-  if (attn_kernel < 0 || attn_kernel > 2 || min_tiles_per_cta < 0) return SPECEXT_ERR_INVALID_ARG;
+  if (attn_kernel < 0 || attn_kernel > 3 || min_tiles_per_cta < 0) return SPECEXT_ERR_INVALID_ARG;
   g_attn_kernel.store(attn_kernel);
   if (min_tiles_per_cta > 0) g_min_units.store(min_tiles_per_cta);
   return SPECEXT_OK;

@@ -1,0 +1,724 @@
+// Hybrid Tree Attention on pairs of SMs (tcgen05 cta_group::2), head dimension 128, row blocks of
+// 256 stacked query rows.
+//
+// A cluster of two CTAs works on one range of (problem, 128-key tile) units.  CTA r of the pair
+// owns the 128 query rows r*128.. of the row block: its Q rows, its S tiles, its P and its O
+// accumulator live in its own tensor memory.  Each CTA stages only half of every K/V tile in its
+// shared memory (K: 64 of the 128 keys; V: 64 of the 128 value columns); the pair's MMAs
+// (M = 256, issued by one thread of the leader CTA) read both halves.  Compared with one CTA doing
+// both row tiles this halves the shared-memory traffic per MMA, removes the re-reading of Q from
+// shared memory (Q is the tensor-memory A operand), and frees tensor memory for P buffers of their own:
+//
+//   tensor memory per CTA: O [0,128) | S0 [128,256) | S1 [256,384) | Q [384,448) | P [448,512)
+//
+// A softmax thread pulls its whole S row into registers and releases its S buffer at once, so the
+// S tiles run two key tiles ahead of the exponentials; P is kept in registers until the previous
+// PV has consumed the P buffer, and the PV of a tile is issued whenever its P is complete.  The two softmax warpgroups of a CTA take alternate
+// key tiles of the same 128 rows (one thread per row each); the running reference maximum of a
+// row is handed from tile to tile through shared memory, each warpgroup keeps its own partial row
+// sum, and O is rescaled lazily by whichever warpgroup raises the maximum by more than 2^8.
+//
+// Warps: 0-3 softmax of even tiles, 4-7 softmax of odd tiles, 8 TMA producer (own halves),
+// 9 issuer of the S = Q K^T MMAs and 10 issuer of the O += P V MMAs (leader CTA only; two issuers
+// so that neither kind waits behind the other's barriers), 11 ancestor masks.
+// Barriers with arrivals from both CTAs live in the leader CTA; MMA completion is multicast to
+// both CTAs.  Every wait is bounded; an expired wait raises SPECEXT_ERR_TIMEOUT, and both CTAs
+// always reach the final cluster barrier before tensor memory is freed.
+#include "common.cuh"
+#include "sm100.cuh"
+
+using namespace sm100;
+
+struct Tc2Maps {
+  CUtensorMap kp, vp, kt, vt;
+};
+
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int kProducerWarp = 8, kMmaWarp = 9, kPvWarp = 10, kTreeWarp = 11;
+constexpr int kRegsLaunch = 168, kRegsOther = 64, kRegsSoftmax = 216;
+static_assert(128 * (kRegsLaunch - kRegsOther) >= 256 * (kRegsSoftmax - kRegsLaunch),
+              "setmaxnreg.inc would wait for registers that are never released");
+constexpr int D = 128;
+constexpr int kStageBytes = 16384;             // half of a K tile (64 keys x 128) or of a V tile (128 keys x 64)
+constexpr int kStages = 6;                     // per ring; one ring for K halves, one for V halves
+constexpr int kCtrlOffset = 2 * kStages * kStageBytes;
+constexpr int kSmemBytes = kCtrlOffset + 3072 + 1024;
+constexpr float kRescaleThreshold = 8.0f;      // log2 units
+constexpr uint32_t kColO = 0, kColS = 128, kColQ = 384, kColP = 448;
+
+struct Ctrl {
+  uint64_t k_full[kStages];     // leader: 2 arrivals (one producer per CTA) + bytes of both halves
+  uint64_t k_empty[kStages];    // each CTA: MMA completion, multicast
+  uint64_t v_full[kStages];
+  uint64_t v_empty[kStages];
+  uint64_t q_ready;             // leader: 16 arrivals (every softmax warp of both CTAs)
+  uint64_t s_full[2];           // each CTA: multicast commit; S buffer w holds a tile for warpgroup w
+  uint64_t s_free[2];           // leader: 8 arrivals; warpgroup w of both CTAs has its S tile in registers
+  uint64_t p_full;              // leader: 8 arrivals (the warpgroup of each CTA that produced this tile's P)
+  uint64_t pv_done[2];          // each CTA: multicast commit after the PV of a tile of warpgroup w
+  uint64_t o_done;              // each CTA: multicast commit after the last PV of a segment
+  uint64_t m_pub[2];            // this CTA: 4 arrivals, reference maxima of the tile are published
+  uint64_t drain;
+  uint64_t epi[2];              // this CTA: 8 arrivals, the two meeting points of a segment's epilogue
+  unsigned long long anc[64];
+  int parent[64];
+  float m_row[128];             // reference maximum of each row after the latest tile
+  float l_x[128];               // epilogue: warpgroup 1 hands its row sums to warpgroup 0
+  uint32_t tmem_base;
+  int abort_flag;
+};
+static_assert(sizeof(Ctrl) <= 3072, "control block too large");
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool try_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier of this CTA whose arrivals may come from the peer CTA or from the pair's
+// tensor pipe.  What such a barrier orders is tensor-memory traffic (fenced with tcgen05.fence) and
+// TMA writes (complete_tx), so the default CTA-scope semantics of arrive and wait suffice; cluster-scope
+// release/acquire on every arrival was measurably slower.
+__device__ __forceinline__ bool wait_c(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (try_wait_cluster(bar, parity, 0u)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (try_wait_cluster(bar, parity, 20000u)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+// One arrival for the whole warp: every lane has finished (and fenced) its own work; the warp
+// barrier orders those lanes before lane 0, whose release makes the warp's work visible.
+__device__ __forceinline__ void warp_arrive_cluster(uint32_t cluster_addr, int lane) {
+  __syncwarp();
+  if (lane == 0) arrive_cluster(cluster_addr);
+}
+__device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+}
+// 3-D tiled load into this CTA's shared memory; the completion barrier may be the peer CTA's.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
+      "%5}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+// D[tmem, both CTAs] (+)= A[tmem, own rows of each CTA] * B[smem halves of both CTAs]
+__device__ __forceinline__ void mma_ts_pair(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// One arrival on the barrier at this offset in both CTAs once all MMAs issued so far are complete.
+__device__ __forceinline__ void commit_pair(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+      : "memory");
+}
+
+#ifdef SPX_TRACE
+#define SPX_EVT2(role, idx)                                                                  \
+  do {                                                                                       \
+    if (a.trace && blockIdx.x < 2 && (idx) < 64)                                             \
+      a.trace[((int)blockIdx.x * 12 + (role)) * 64 + (idx)] = clock64() - spx_t_start;       \
+  } while (0)
+#else
+#define SPX_EVT2(role, idx) do {} while (0)
+#endif
+
+template <bool SCORE>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2Maps maps) {
+  const AttnPlan& p = a.plan;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                         ~static_cast<uintptr_t>(1023));
+  unsigned char* ring = base;
+  Ctrl* ctl = reinterpret_cast<Ctrl*>(base + kCtrlOffset);
+  volatile int* abort_flag = &ctl->abort_flag;
+
+#ifdef SPX_TRACE
+  const long long spx_t_start = clock64();
+#endif
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_rank();
+  const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
+  const int unit_lo = spx_unit_start(p, cl), unit_hi = spx_unit_start(p, cl + 1);
+
+  if (warp == kProducerWarp && lane == 0) {
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&ctl->k_full[i], 2);
+      mbar_init(&ctl->k_empty[i], 1);
+      mbar_init(&ctl->v_full[i], 2);
+      mbar_init(&ctl->v_empty[i], 1);
+    }
+    mbar_init(&ctl->q_ready, 16);      // one arrival per softmax warp of both CTAs
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ctl->s_full[i], 1);
+      mbar_init(&ctl->s_free[i], 8);    // one arrival per warp: 4 warps of the warpgroup x 2 CTAs
+      mbar_init(&ctl->pv_done[i], 1);
+      mbar_init(&ctl->m_pub[i], 4);
+    }
+    mbar_init(&ctl->p_full, 8);
+    mbar_init(&ctl->o_done, 1);
+    mbar_init(&ctl->drain, 2);
+    mbar_init(&ctl->epi[0], 8);
+    mbar_init(&ctl->epi[1], 8);
+    ctl->abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tensormap(&maps.kp);
+    prefetch_tensormap(&maps.vp);
+    prefetch_tensormap(&maps.kt);
+    prefetch_tensormap(&maps.vt);
+  }
+  cluster_sync_all();                    // both CTAs' barriers exist before anyone signals them
+  bool ok = true;
+
+  if (warp == kProducerWarp) {
+    // ================================ TMA producer (each CTA loads its halves) ===============
+    setmaxnreg_dec<kRegsOther>();
+    if (lane == 0) {
+      uint32_t kp = 0, vp = 0;
+      const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
+      const uint32_t vfull0 = map_to_cta(smem_u32(&ctl->v_full[0]), 0);
+      for (int u = unit_lo; u < unit_hi && ok;) {
+        const int prob = u / p.UPP;
+        const int tile_lo = u - prob * p.UPP;
+        const int n = min(p.UPP - tile_lo, unit_hi - u);
+        const int g = prob / p.n_rblk;
+        for (int j = 0; j < n && ok; ++j) {
+          const int tile = tile_lo + j;
+          const bool is_tree = tile == p.TPH;
+          {   // K half: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
+            const int stage = kp % kStages;
+            ok = wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            const uint32_t bar = kfull0 + stage * 8;
+            const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+            const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
+            const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
+            arrive_expect_tx_cluster(bar, kStageBytes);
+            tma_load_3d_pair(dst, m, bar, 0, g, key0);
+            tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
+            SPX_EVT2(0, 2 * j);
+            ++kp;
+          }
+          {   // V half: value columns [64*rank, 64*rank+64) of all 128 keys
+            const int stage = vp % kStages;
+            ok = wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            const uint32_t bar = vfull0 + stage * 8;
+            const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
+            arrive_expect_tx_cluster(bar, kStageBytes);
+            tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
+            SPX_EVT2(0, 2 * j + 1);
+            ++vp;
+          }
+        }
+        u += n;
+      }
+    }
+  } else {
+    if (warp == kMmaWarp) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                   "r"(512u)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else if (warp == kTreeWarp) {
+      ctl->parent[lane] = lane < p.T ? a.parent[lane] : -1;
+      ctl->parent[lane + 32] = lane + 32 < p.T ? a.parent[lane + 32] : -1;
+      __syncwarp();
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int t = lane + 32 * half;
+        unsigned long long m = 0;
+        if (t < p.T) {
+          int u = t;
+          for (int step = 0; step <= p.T && u >= 0; ++step) {
+            m |= 1ull << u;
+            const int pu = ctl->parent[u];
+            if (pu < -1 || pu >= u) {
+              if (blockIdx.x == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
+              break;
+            }
+            u = pu;
+          }
+        }
+        ctl->anc[t] = m;
+      }
+    }
+    tc_fence_before();
+    named_bar_sync(1, kThreads - 32);
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+
+    if (warp == kMmaWarp) {
+      // ================================ issuer of S = Q K^T (leader CTA) =====================
+      setmaxnreg_dec<kRegsOther>();
+      if (lane == 0 && rank == 0) {
+        const uint32_t idesc_s = idesc_bf16_f32(256, SPX_TILE_KEYS, false, false);
+        constexpr uint32_t hi = desc_hi(1024);
+        const uint32_t ring_lo = desc_lo(smem_u32(ring), 16);
+        uint32_t kc = 0, n_w[2] = {0, 0};          // n_w[w]: S tiles issued so far for warpgroup w
+        int seg = 0;
+        for (int u = unit_lo; u < unit_hi && ok;) {
+          const int prob = u / p.UPP;
+          const int tile_lo = u - prob * p.UPP;
+          const int n = min(p.UPP - tile_lo, unit_hi - u);
+          ok = wait_c(&ctl->q_ready, seg & 1, abort_flag);
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            // S buffer w is free once warpgroup w holds its previous tile in registers
+            if (n_w[w] > 0) ok = wait_c(&ctl->s_free[w], (n_w[w] - 1) & 1, abort_flag);
+            const int stage = kc % kStages;
+            if (ok) ok = wait_c(&ctl->k_full[stage], (kc / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t kb = ring_lo + stage * (kStageBytes >> 4);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk)
+              mma_ts_pair(tmem + kColS + w * 128, tmem + kColQ + kk * 8, kb + (kk >> 2) * 512 + (kk & 3) * 2, hi,
+                          idesc_s, kk > 0 ? 1u : 0u);
+            commit_pair(&ctl->s_full[w]);
+            commit_pair(&ctl->k_empty[stage]);
+            SPX_EVT2(1, j);
+            ++kc;
+            ++n_w[w];
+          }
+          u += n;
+          ++seg;
+        }
+        commit_pair(&ctl->drain);
+      }
+    } else if (warp == kPvWarp) {
+      // ================================ issuer of O += P V (leader CTA) ======================
+      setmaxnreg_dec<kRegsOther>();
+      if (lane == 0 && rank == 0) {
+        const uint32_t idesc_o = idesc_bf16_f32(256, D, false, true);
+        constexpr uint32_t hi = desc_hi(1024);
+        const uint32_t ring_lo = desc_lo(smem_u32(ring + kStages * kStageBytes), 16);
+        uint32_t vc = 0;                           // V tiles consumed = PVs issued
+        int seg = 0;
+        for (int u = unit_lo; u < unit_hi && ok;) {
+          const int prob = u / p.UPP;
+          const int tile_lo = u - prob * p.UPP;
+          const int n = min(p.UPP - tile_lo, unit_hi - u);
+          ok = wait_c(&ctl->q_ready, seg & 1, abort_flag);      // every thread is done reading the previous O
+          for (int j = 0; j < n && ok; ++j) {
+            const int w = j & 1;
+            const int stage = vc % kStages;
+            ok = wait_c(&ctl->v_full[stage], (vc / kStages) & 1, abort_flag);
+            if (ok) ok = wait_c(&ctl->p_full, vc & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            SPX_EVT2(11, 2 * j);
+            const uint32_t vb = ring_lo + stage * (kStageBytes >> 4);
+            const uint32_t pa = tmem + kColP;
+            mma_ts_pair(tmem + kColO, pa, vb, hi, idesc_o, j > 0 ? 1u : 0u);
+#pragma unroll
+            for (int kk = 1; kk < SPX_TILE_KEYS / 16; ++kk)
+              mma_ts_pair(tmem + kColO, pa + kk * 8, vb + kk * 128, hi, idesc_o, 1u);
+            commit_pair(&ctl->v_empty[stage]);
+            commit_pair(&ctl->pv_done[w]);
+            if (j == n - 1) commit_pair(&ctl->o_done);
+            SPX_EVT2(11, 2 * j + 1);
+            ++vc;
+          }
+          u += n;
+          ++seg;
+        }
+        commit_pair(&ctl->drain);
+        // everything issued by both issuers must be complete before tensor memory is released
+        for (int spin = 0; spin < (1 << 22) && !try_wait_cluster(&ctl->drain, 0, 0u); ++spin) {}
+      }
+    } else if (warp == kTreeWarp) {
+      setmaxnreg_dec<kRegsOther>();
+    } else {
+      // ================================ softmax warps =======================================
+      setmaxnreg_inc<kRegsSoftmax>();
+      const int wg = warp >> 2;                          // 0: even tiles, 1: odd tiles
+      const int quarter = warp & 3;
+      const int row_t = quarter * 32 + lane;             // row inside this CTA's 128-row tile
+      const int rr = rank * 128 + row_t;                 // row inside the 256-row block
+      const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+      const uint32_t s_addr = tmem + lane_addr + kColS + wg * 128;
+      const uint32_t p_addr = tmem + lane_addr + kColP;
+      const uint32_t o_addr = tmem + lane_addr + kColO;
+      const uint32_t q_ready_l = map_to_cta(smem_u32(&ctl->q_ready), 0);
+      const uint32_t p_full_l = map_to_cta(smem_u32(&ctl->p_full), 0);
+      const uint32_t s_free_l = map_to_cta(smem_u32(&ctl->s_free[wg]), 0);
+      const float scale2 = p.scale2;
+      uint32_t n_mine = 0;       // tiles this warpgroup has processed (phase of s_full[wg], m_pub[wg])
+      uint32_t n_other = 0;      // tiles of the other warpgroup whose maxima this one has consumed
+      uint32_t n_oth = 0;        // tiles the other warpgroup had been given before the current segment
+      int seg = 0;
+      for (int u = unit_lo; u < unit_hi && ok;) {
+        const int prob = u / p.UPP;
+        const int tile_lo = u - prob * p.UPP;
+        const int n = min(p.UPP - tile_lo, unit_hi - u);
+        const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+        const int r = rblk * p.RB + rr;
+        const bool valid = r < p.rows;
+        const int t_node = valid ? r / p.G : 0;
+        const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
+
+        // Q row of this thread -> tensor memory (warpgroup 0: first 64 elements, warpgroup 1: the rest)
+        {
+          uint32_t qv[32];
+          if (valid) {
+            const uint4* qp = reinterpret_cast<const uint4*>(a.Q + (long long)t_node * a.q_st +
+                                                             (long long)(g * p.G + r % p.G) * a.q_sh + wg * 64);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint4 x = __ldg(qp + j);
+              qv[j * 4] = x.x; qv[j * 4 + 1] = x.y; qv[j * 4 + 2] = x.z; qv[j * 4 + 3] = x.w;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) qv[j] = 0u;
+          }
+          tmem_st32(tmem + lane_addr + kColQ + wg * 32, qv);
+          tmem_wait_st();
+          tc_fence_before();
+          warp_arrive_cluster(q_ready_l, lane);
+        }
+
+        float m_loc = -INFINITY, l = 0.f;        // l is relative to m_loc
+        for (int j = wg; j < n && ok; j += 2) {
+          const int tile = tile_lo + j;
+          const bool is_tree = tile == p.TPH;
+          const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
+          const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
+          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1));
+          ok = wait_c(&ctl->s_full[wg], n_mine & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 1);
+          uint32_t s0[32], s1[32], s2[32], s3[32];
+          tmem_ld32(s_addr, s0);
+          tmem_ld32(s_addr + 32, s1);
+          tmem_ld32(s_addr + 64, s2);
+          tmem_ld32(s_addr + 96, s3);
+          tmem_wait_ld();
+          tc_fence_before();
+          warp_arrive_cluster(s_free_l, lane);          // the S buffer may take the next tile
+          if (need_mask) {
+            unsigned long long vis_lo, vis_hi;
+            if (is_tree) {
+              vis_lo = tree_mask;
+              vis_hi = 0ull;
+            } else {
+              vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
+              vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);
+            }
+            const uint32_t b0 = static_cast<uint32_t>(vis_lo), b1 = static_cast<uint32_t>(vis_lo >> 32);
+            const uint32_t b2 = static_cast<uint32_t>(vis_hi), b3 = static_cast<uint32_t>(vis_hi >> 32);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) {
+              if (!((b0 >> k) & 1u)) s0[k] = 0xff800000u;    // -inf
+              if (!((b1 >> k) & 1u)) s1[k] = 0xff800000u;
+              if (!((b2 >> k) & 1u)) s2[k] = 0xff800000u;
+              if (!((b3 >> k) & 1u)) s3[k] = 0xff800000u;
+            }
+          }
+          float t0 = -INFINITY, t1 = -INFINITY, t2 = -INFINITY, t3 = -INFINITY;
+#pragma unroll
+          for (int k = 0; k < 32; k += 2) {
+            t0 = fmax3(t0, __uint_as_float(s0[k]), __uint_as_float(s0[k + 1]));
+            t1 = fmax3(t1, __uint_as_float(s1[k]), __uint_as_float(s1[k + 1]));
+            t2 = fmax3(t2, __uint_as_float(s2[k]), __uint_as_float(s2[k + 1]));
+            t3 = fmax3(t3, __uint_as_float(s3[k]), __uint_as_float(s3[k + 1]));
+          }
+          const float m_tile = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * scale2;
+
+          // the row's reference maximum after the previous tile (handled by the other warpgroup)
+          float m_cur = -INFINITY;
+          if (j > 0) {
+            ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
+            if (!ok) break;
+            ++n_other;
+            m_cur = ctl->m_row[row_t];
+          }
+          float m_new = m_cur;
+          bool rescale = false;
+          if (m_tile > m_cur + kRescaleThreshold || m_cur == -INFINITY) {
+            m_new = m_tile;
+            rescale = j > 0;
+          }
+          ctl->m_row[row_t] = m_new;
+          warp_arrive(&ctl->m_pub[wg], lane);
+          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 2);
+          if (m_loc != m_new) {
+            l *= (m_loc == -INFINITY) ? 0.f : ex2_approx(m_loc - m_new);
+            m_loc = m_new;
+          }
+          // Completion of the PV of tile j-1 (the other warpgroup's) is needed before O may be
+          // rescaled and before the P buffer may be overwritten.  The PV of this warpgroup's own
+          // previous tile (j-2) is waited for first: once it is complete so is every earlier one,
+          // which keeps the parity test on the other barrier unambiguous.
+          const uint32_t n_prev_other = n_oth + ((j + 1) >> 1);      // tiles given to the other warpgroup before j
+          bool pv_seen = false;
+          auto wait_prev_pv = [&]() -> bool {
+            if (pv_seen) return true;
+            pv_seen = true;
+            if (n_mine > 0 && !wait_c(&ctl->pv_done[wg], (n_mine - 1) & 1, abort_flag)) return false;
+            if (n_prev_other > 0 && !wait_c(&ctl->pv_done[wg ^ 1], (n_prev_other - 1) & 1, abort_flag)) return false;
+            tc_fence_after();
+            return true;
+          };
+          if (__any_sync(0xffffffffu, rescale)) {
+            // O must hold the sum up to tile j-1 and nothing may be accumulating into it
+            ok = wait_prev_pv();
+            if (!ok) break;
+            const float alpha = rescale ? ex2_approx(m_cur - m_new) : 1.f;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t v[32];
+              tmem_ld32(o_addr + c * 32, v);
+              tmem_wait_ld();
+#pragma unroll
+              for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(__uint_as_float(v[k]) * alpha);
+              tmem_st32(o_addr + c * 32, v);
+            }
+          }
+
+          const float neg_m = -m_new;
+          const bool score = SCORE && !is_tree;
+          float* mass = nullptr;
+          if (score) {
+            const long long rowbase = ((long long)prob * p.TPH + tile) * p.RB + rr;
+            mass = a.ws + p.off_mass + rowbase * p.CPT;
+            a.ws[p.off_mref + rowbase] = m_new;
+          }
+          float csum = 0.f;
+          uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
+          auto exp_chunk = [&](uint32_t (&v)[32], uint32_t (&pk)[16], int c) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k)
+              v[k] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(v[k]), scale2, neg_m)));
+            float gs0 = 0.f, gs1 = 0.f, gs2 = 0.f, gs3 = 0.f;
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+              gs0 += __uint_as_float(v[k]);
+              gs1 += __uint_as_float(v[k + 1]);
+              gs2 += __uint_as_float(v[k + 2]);
+              gs3 += __uint_as_float(v[k + 3]);
+            }
+            const float gs = (gs0 + gs1) + (gs2 + gs3);
+            l += gs;
+            if (score) {
+              if (p.C >= 32) {
+                csum += gs;
+                if ((((c + 1) * 32) & (p.C - 1)) == 0) {
+                  mass[((c + 1) * 32) / p.C - 1] = csum;
+                  csum = 0.f;
+                }
+              } else {
+                float acc = 0.f;
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                  acc += __uint_as_float(v[k]);
+                  if (((k + 1) & (p.C - 1)) == 0) {
+                    mass[(c * 32 + k) / p.C] = acc;
+                    acc = 0.f;
+                  }
+                }
+              }
+            }
+#pragma unroll
+            for (int k = 0; k < 16; ++k) pk[k] = pack_bf16x2(__uint_as_float(v[2 * k]), __uint_as_float(v[2 * k + 1]));
+          };
+          exp_chunk(s0, pk0, 0);
+          exp_chunk(s1, pk1, 1);
+          exp_chunk(s2, pk2, 2);
+          exp_chunk(s3, pk3, 3);
+          // the P buffer is shared by all tiles: the PV of the previous tile must have read it
+          ok = wait_prev_pv();
+          if (!ok) break;
+          tmem_st16(p_addr, pk0);
+          tmem_st16(p_addr + 16, pk1);
+          tmem_st16(p_addr + 32, pk2);
+          tmem_st16(p_addr + 48, pk3);
+          tmem_wait_st();
+          tc_fence_before();
+          warp_arrive_cluster(p_full_l, lane);
+          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 3);
+          ++n_mine;
+        }
+        if (!ok) break;
+
+        // ---- epilogue of the segment --------------------------------------------------------
+        // final reference maximum: published by the warpgroup that handled the last tile
+        if (((n - 1) & 1) != wg) {
+          ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
+          if (!ok) break;
+          ++n_other;
+        }
+        const float m_fin = ctl->m_row[row_t];
+        if (m_loc != m_fin) l *= (m_loc == -INFINITY) ? 0.f : ex2_approx(m_loc - m_fin);
+        if (wg == 1) ctl->l_x[row_t] = l;
+        if (lane == 0) SPX_EVT2(2 + warp, 60);
+        ok = wait_c(&ctl->o_done, seg & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) SPX_EVT2(2 + warp, 61);
+        n_oth += wg == 0 ? (n >> 1) : ((n + 1) >> 1);
+        warp_arrive(&ctl->epi[0], lane);                 // l_x visible; both warpgroups past their last tile
+        ok = mbar_wait(&ctl->epi[0], seg & 1, abort_flag);
+        if (!ok) break;
+        {
+          const int slot = cl + prob;
+          float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {                  // this warpgroup's 64 of the 128 columns
+            uint32_t v[32];
+            tmem_ld32(o_addr + wg * 64 + c * 32, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 x = make_float4(__uint_as_float(v[q4 * 4]), __uint_as_float(v[q4 * 4 + 1]),
+                                           __uint_as_float(v[q4 * 4 + 2]), __uint_as_float(v[q4 * 4 + 3]));
+              *reinterpret_cast<float4*>(po + ((long long)(wg * 16 + c * 8 + q4) * p.RB + rr) * 4) = x;
+            }
+          }
+          if (wg == 0) {
+            a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_fin;
+            a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l + ctl->l_x[row_t];
+          }
+        }
+        if (lane == 0) SPX_EVT2(2 + warp, 62);
+        warp_arrive(&ctl->epi[1], lane);                 // l_x and m_row may be reused
+        ok = mbar_wait(&ctl->epi[1], seg & 1, abort_flag);
+        ++seg;
+        u += n;
+      }
+    }
+  }
+
+  if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
+  tc_fence_before();
+  if (tid == 0) SPX_EVT2(10, 0);
+  cluster_sync_all();
+  if (tid == 0) SPX_EVT2(10, 1);                    // the peer may still signal this CTA's barriers or read its halves
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(ctl->tmem_base), "r"(512u) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn2() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 tensor [n2][n1][128] with element strides (s2, s1, 1); box = 64 x 1 x b2, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_map2(CUtensorMap* m, const void* ptr, long long n1, long long s1, long long n2, long long s2, int b2) {
+  EncodeTiledFn fn = encode_fn2();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)n1, (cuuint64_t)n2};
+  const cuuint64_t strides[2] = {(cuuint64_t)s1 * 2, (cuuint64_t)s2 * 2};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)b2};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool SCORE>
+cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel<SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * a.plan.n_cta);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attn_tc2_kernel<SCORE>, a, maps);
+}
+
+}  // namespace
+
+// Requires head_dim 128 and 256-row blocks (plan.RB == 256); plan.n_cta counts clusters of two CTAs.
+cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launches) {
+  const AttnPlan& p = a.plan;
+  if (p.D != D || p.RB != 256) return cudaErrorInvalidValue;
+  Tc2Maps maps;
+  bool ok = encode_map2(&maps.kt, a.Kt, p.Hkv, a.tkv_sh, p.T, a.tkv_st, 64);
+  ok = ok && encode_map2(&maps.vt, a.Vt, p.Hkv, a.tkv_sh, p.T, a.tkv_st, SPX_TILE_KEYS);
+  if (p.L > 0) {
+    ok = ok && encode_map2(&maps.kp, a.Kp, p.Hkv, a.kv_sh, p.L, a.kv_sl, 64);
+    ok = ok && encode_map2(&maps.vp, a.Vp, p.Hkv, a.kv_sh, p.L, a.kv_sl, SPX_TILE_KEYS);
+  } else {
+    maps.kp = maps.kt;
+    maps.vp = maps.vt;
+  }
+  if (!ok) return cudaErrorInvalidValue;
+  const cudaError_t e = p.want_score ? launch2<true>(a, maps, st) : launch2<false>(a, maps, st);
+  *n_launches += 1;
+  return e;
+}

@@ -69,6 +69,7 @@ __device__ __forceinline__ void spx_build_ancestors(const int32_t* __restrict__ 
 // Launchers implemented in the kernel translation units; each returns the cudaError_t of its launch.
 cudaError_t spx_launch_attn_simt(const AttnArgs& a, cudaStream_t st, int* n_launches);
 cudaError_t spx_launch_attn_tc(const AttnArgs& a, cudaStream_t st, int* n_launches);
+cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launches);
 cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches);
 
 #endif  // SPECEXT_COMMON_CUH_

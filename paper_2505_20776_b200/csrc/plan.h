@@ -7,10 +7,13 @@
 // Units.  The prefix is cut into key tiles of 128 tokens; the tree keys form one more tile.  A
 // problem therefore has UPP = ceil(L/128) + 1 units, the last one being the tree tile.  All
 // units of all problems are laid out in one line (problem-major) and cut into n_cta contiguous
-// ranges of nearly equal length; CTA c owns units [unit_start(c), unit_start(c+1)).  The part of
-// a CTA's range that lies inside one problem is a "segment" and yields one partial result
-// (unnormalised output, running maximum, row sum) in slot c + problem.  Slots are unique because
-// both c and the problem index are non-decreasing along the line.
+// ranges; worker c (a CTA, or a cluster of two CTAs for the paired kernel) owns units
+// [unit_start(c), unit_start(c+1)).  With cpp > 0 every problem gets the same whole number cpp of
+// workers and its units are spread evenly over them, so that no worker straddles two problems;
+// with cpp == 0 the whole line is cut into n_cta nearly equal ranges.  The part of a worker's
+// range that lies inside one problem is a "segment" and yields one partial result (unnormalised
+// output, running maximum, row sum) in slot c + problem.  Slots are unique because both c and the
+// problem index are non-decreasing along the line.
 #ifndef SPECEXT_PLAN_H_
 #define SPECEXT_PLAN_H_
 
@@ -33,8 +36,10 @@ struct AttnPlan {
   int TPH;         // prefix key tiles per problem = ceil(L/128)
   int UPP;         // units per problem = TPH + 1 (tree tile last)
   int U;           // total units
-  int n_cta;       // CTAs of the attention kernel (<= U)
-  int q, rem;      // U = q*n_cta + rem
+  int n_cta;       // workers of the attention kernel (<= U)
+  int kernel;      // 1 CUDA-core kernel, 2 one-CTA tensor-core kernel, 3 paired-CTA tensor-core kernel
+  int cpp;         // workers per problem, or 0 when the line of units is cut without regard to problems
+  int q, rem;      // cpp > 0: UPP = q*cpp + rem;  cpp == 0: U = q*n_cta + rem
   int n_slots;     // n_cta + NP - 1 partial slots
   int max_segs;    // upper bound on segments per problem
   int CPT;         // chunks per key tile = 128 / C
@@ -45,11 +50,21 @@ struct AttnPlan {
   long long off_part_o, off_part_m, off_part_l, off_mass, off_mref, total_floats;
 };
 
-SPX_HD int spx_unit_start(const AttnPlan& p, int c) { return c * p.q + (c < p.rem ? c : p.rem); }
+SPX_HD int spx_unit_start(const AttnPlan& p, int c) {
+  if (p.cpp > 0) {
+    const int prob = c / p.cpp, k = c - prob * p.cpp;
+    return prob * p.UPP + k * p.q + (k < p.rem ? k : p.rem);
+  }
+  return c * p.q + (c < p.rem ? c : p.rem);
+}
 
-// CTA that owns unit u.
+// Worker that owns unit u.
 SPX_HD int spx_unit_owner(const AttnPlan& p, int u) {
   const int big = p.rem * (p.q + 1);
+  if (p.cpp > 0) {
+    const int prob = u / p.UPP, w = u - prob * p.UPP;
+    return prob * p.cpp + (w < big ? w / (p.q + 1) : p.rem + (w - big) / p.q);
+  }
   return u < big ? u / (p.q + 1) : p.rem + (u - big) / p.q;
 }
 

@@ -50,13 +50,13 @@ def test_static_scratch_entry_matches_the_ordinary_one(cuda_device):
 
 def test_static_scratch_entry_rejects_what_does_not_fit(cuda_device):
     dev = cuda_device
-    w = synth.WORKLOADS["c3"]                                      # 64K prefix with scores: > 32 MiB of scratch
+    w = synth.WORKLOADS["c3"]                                      # 256K prefix with scores: > 32 MiB of scratch
     t = {k: v.to(dev) for k, v in synth.make_layer(w.with_prefix(256), capacity=256).items()}
     O = torch.empty_like(t["Q"])
-    d = api.make_attn_desc(t["Q"], t["K_prefix"], t["K_tree"], O, 65536, w.chunk_size, 0.0, True)
+    d = api.make_attn_desc(t["Q"], t["K_prefix"], t["K_tree"], O, 1 << 18, w.chunk_size, 0.0, True)
     assert api.specext_verify_attn_workspace(d) > api.STATIC_SCRATCH_BYTES
     lse = torch.empty(w.n_q_heads, w.n_tree, dtype=torch.float32, device=dev)
-    cs = torch.empty(w.n_tree, 2048, dtype=torch.float32, device=dev)
+    cs = torch.empty(w.n_tree, 8192, dtype=torch.float32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     parent = torch.from_numpy(synth.make_tree(w)).to(dev)
     with pytest.raises(api.SpecextError) as e:
