@@ -61,6 +61,7 @@ struct Ctrl {
   uint64_t o_done;              // each CTA: multicast commit after the last PV of a segment
   uint64_t m_pub[2];            // this CTA: 4 arrivals, reference maxima of the tile are published
   uint64_t drain;
+  uint64_t anc_ready;           // this CTA: the ancestor masks are in shared memory
   uint64_t epi[2];              // this CTA: 8 arrivals, the two meeting points of a segment's epilogue
   unsigned long long anc[64];
   int parent[64];
@@ -204,6 +205,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     mbar_init(&ctl->p_full, 8);
     mbar_init(&ctl->o_done, 1);
     mbar_init(&ctl->drain, 2);
+    mbar_init(&ctl->anc_ready, 1);
     mbar_init(&ctl->epi[0], 8);
     mbar_init(&ctl->epi[1], 8);
     ctl->abort_flag = 0;
@@ -231,6 +233,13 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         for (int j = 0; j < n && ok; ++j) {
           const int tile = tile_lo + j;
           const bool is_tree = tile == p.TPH;
+          // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A
+          // full ring requested at once by every SM sits in the memory system's queues in no
+          // particular order, and tile 0 would arrive last as often as first.
+          if (kp == 2) {
+            ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
+            if (!ok) break;
+          }
           {   // K half: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
             const int stage = kp % kStages;
             ok = wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag);
@@ -267,6 +276,8 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
                    : "memory");
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     } else if (warp == kTreeWarp) {
+      // registers first: the softmax warpgroups cannot grow until every warp of this warpgroup has shrunk
+      setmaxnreg_dec<kRegsOther>();
       ctl->parent[lane] = lane < p.T ? a.parent[lane] : -1;
       ctl->parent[lane + 32] = lane + 32 < p.T ? a.parent[lane + 32] : -1;
       __syncwarp();
@@ -288,9 +299,11 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         }
         ctl->anc[t] = m;
       }
+      warp_arrive(&ctl->anc_ready, lane);
     }
+    // the tensor-memory base address is visible to everybody who uses it (not the producer, not the tree warp)
     tc_fence_before();
-    named_bar_sync(1, kThreads - 32);
+    if (warp != kTreeWarp) named_bar_sync(1, kThreads - 64);
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
 
@@ -374,7 +387,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         for (int spin = 0; spin < (1 << 22) && !try_wait_cluster(&ctl->drain, 0, 0u); ++spin) {}
       }
     } else if (warp == kTreeWarp) {
-      setmaxnreg_dec<kRegsOther>();
+      // nothing left to do
     } else {
       // ================================ softmax warps =======================================
       setmaxnreg_inc<kRegsSoftmax>();
@@ -402,6 +415,10 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const int r = rblk * p.RB + rr;
         const bool valid = r < p.rows;
         const int t_node = valid ? r / p.G : 0;
+        if (seg == 0) {
+          ok = mbar_wait(&ctl->anc_ready, 0, abort_flag);
+          if (!ok) break;
+        }
         const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
 
         // Q row of this thread -> tensor memory (warpgroup 0: first 64 elements, warpgroup 1: the rest)

@@ -40,22 +40,29 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   const float* po = a.ws + p.off_part_o + (((long long)slot0 * nd4 + d4) * p.RB + rr) * 4;
   const long long ostride = (long long)nd4 * p.RB * 4;
 
-  float M = -INFINITY;
-  for (int s = 0; s < nseg; ++s) M = fmaxf(M, pm[(long long)s * p.RB]);
-  float Z = 0.f;
+  // Batches of 8 segments with every load of a batch in flight at once (the loads of one thread are
+  // independent; issued one by one they would each pay the full memory latency).
+  float M = -INFINITY, Z = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  int s = 0;
-  for (; s + 4 <= nseg; s += 4) {
-    float ms[4], ls[4];
-    float4 v[4];
+  for (int s = 0; s < nseg; s += 8) {
+    float ms[8], ls[8];
+    float4 v[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      ms[k] = pm[(long long)(s + k) * p.RB];
-      ls[k] = pl[(long long)(s + k) * p.RB];
-      v[k] = *reinterpret_cast<const float4*>(po + (s + k) * ostride);
+    for (int k = 0; k < 8; ++k) {
+      const bool in = s + k < nseg;
+      ms[k] = in ? __ldcg(pm + (long long)(s + k) * p.RB) : -INFINITY;
+      ls[k] = in ? __ldcg(pl + (long long)(s + k) * p.RB) : 0.f;
+      v[k] = in ? __ldcg(reinterpret_cast<const float4*>(po + (s + k) * ostride)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    float Mb = M;
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < 8; ++k) Mb = fmaxf(Mb, ms[k]);
+    const float carry = exp2f(M - Mb);              // 0 on the first batch (M = -inf)
+    Z *= carry;
+    acc.x *= carry; acc.y *= carry; acc.z *= carry; acc.w *= carry;
+    M = Mb;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
       const float w = exp2f(ms[k] - M);
       Z = fmaf(ls[k], w, Z);
       acc.x = fmaf(w, v[k].x, acc.x);
@@ -63,15 +70,6 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
       acc.z = fmaf(w, v[k].z, acc.z);
       acc.w = fmaf(w, v[k].w, acc.w);
     }
-  }
-  for (; s < nseg; ++s) {
-    const float w = exp2f(pm[(long long)s * p.RB] - M);
-    const float4 v = *reinterpret_cast<const float4*>(po + s * ostride);
-    Z = fmaf(pl[(long long)s * p.RB], w, Z);
-    acc.x = fmaf(w, v.x, acc.x);
-    acc.y = fmaf(w, v.y, acc.y);
-    acc.z = fmaf(w, v.z, acc.z);
-    acc.w = fmaf(w, v.w, acc.w);
   }
   const float inv = 1.f / Z;
   const int t = r / p.G, h = g * p.G + r % p.G;
