@@ -393,3 +393,24 @@ def test_coarser_splits_give_the_same_result(cuda_device):
         check_attn(hp, t_cpu, parent, w.prefix_len, w.chunk_size)
     finally:
         api.specext_set_tuning(0, 1)
+
+
+def test_one_cta_kernel_on_a_paired_kernel_shape(cuda_device):
+    """The one-CTA tensor-core kernel stays correct for shapes that default to the paired kernel."""
+    w = synth.WORKLOADS["c1"]
+    try:
+        api.specext_set_tuning(2, 0)
+        hp = make_hp(w, cuda_device)
+        check_attn(hp, synth.make_layer(w), synth.make_tree(w), w.prefix_len, w.chunk_size)
+    finally:
+        api.specext_set_tuning(0, 0)
+
+
+def test_paired_kernel_with_more_problems_than_clusters(cuda_device):
+    """80 KV heads > 74 clusters: every cluster works through several (KV head) segments."""
+    w = _small(320, 80, 128, 200, 40, 32)
+    hp = make_hp(w, cuda_device)
+    check_attn(hp, synth.make_layer(w), synth.make_tree(w), 200, 32)
+    w = _small(160, 80, 128, 96, 64, 32)          # rows = 128 -> one-CTA kernel, one short tile, many problems
+    hp = make_hp(w, cuda_device)
+    check_attn(hp, synth.make_layer(w), synth.make_tree(w), 96, 32)
