@@ -188,6 +188,36 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
   const int unit_lo = spx_unit_start(p, cl), unit_hi = spx_unit_start(p, cl + 1);
 
+  // The first segment's Q rows are requested before anything else, with asynchronous copies into a
+  // shared-memory scratch, so that their latency (a first touch of the page costs a TLB miss on top
+  // of DRAM) runs under the set-up instead of delaying the first S MMA.  8 lanes copy the 128 bytes
+  // a thread needs of one row (warpgroup 0: first 64 elements, warpgroup 1: the rest); 16-byte chunks
+  // are XOR-swizzled by the row so that the copies and the later per-row reads are conflict-free.
+  // The scratch (4 KB per warp) is the tail of the V ring, which the producer leaves alone until
+  // the first S MMA is done.
+  if (warp < kProducerWarp && unit_lo < unit_hi) {
+    const int prob = unit_lo / p.UPP;
+    const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+    const int r0 = rblk * p.RB + (int)rank * 128 + (warp & 3) * 32;
+    const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + (warp >> 2) * 64;
+    unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int row = it * 4 + (lane >> 3), rw = r0 + row;
+      unsigned char* dst = scratch + row * 128 + (((lane & 7) ^ (row & 7)) << 4);
+      if (rw < p.rows) {
+        const __nv_bfloat16* src = qbase + (long long)(rw / p.G) * a.q_st + (long long)(rw % p.G) * a.q_sh + (lane & 7) * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  } else if (warp == kTreeWarp && lane == 0) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.parent));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.parent + 32));
+  }
+
   if (warp == kProducerWarp && lane == 0) {
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&ctl->k_full[i], 2);
@@ -224,6 +254,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     if (lane == 0) {
       uint32_t kp = 0, vp = 0;
       const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
+
       const uint32_t vfull0 = map_to_cta(smem_u32(&ctl->v_full[0]), 0);
       for (int u = unit_lo; u < unit_hi && ok;) {
         const int prob = u / p.UPP;
@@ -424,9 +455,22 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         // Q row of this thread -> tensor memory (warpgroup 0: first 64 elements, warpgroup 1: the rest)
         {
           uint32_t qv[32];
-          if (valid) {
-            const uint4* qp = reinterpret_cast<const uint4*>(a.Q + (long long)t_node * a.q_st +
-                                                             (long long)(g * p.G + r % p.G) * a.q_sh + wg * 64);
+          const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + wg * 64;
+          if (seg == 0) {
+            // requested at kernel start (see above)
+            const unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint4 y = *reinterpret_cast<const uint4*>(scratch + lane * 128 + ((j ^ (lane & 7)) << 4));
+              qv[j * 4] = y.x; qv[j * 4 + 1] = y.y; qv[j * 4 + 2] = y.z; qv[j * 4 + 3] = y.w;
+            }
+            // the scratch goes back to the V ring, which the TMA unit writes
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          } else if (valid) {
+            const uint4* qp = reinterpret_cast<const uint4*>(qbase + (long long)t_node * a.q_st +
+                                                             (long long)(r % p.G) * a.q_sh);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const uint4 x = __ldg(qp + j);
