@@ -218,32 +218,40 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.parent + 32));
   }
 
-  if (warp == kProducerWarp && lane == 0) {
-    for (int i = 0; i < kStages; ++i) {
-      mbar_init(&ctl->k_full[i], 2);
-      mbar_init(&ctl->k_empty[i], 1);
-      mbar_init(&ctl->v_full[i], 2);
-      mbar_init(&ctl->v_empty[i], 1);
-    }
-    mbar_init(&ctl->q_ready, 16);      // one arrival per softmax warp of both CTAs
-    for (int i = 0; i < 2; ++i) {
+  if (warp == kProducerWarp) {
+    // one barrier per lane (the four ring arrays first), so that the set-up is not 40 serial inits
+    if (lane < kStages) {
+      mbar_init(&ctl->k_full[lane], 2);
+      mbar_init(&ctl->k_empty[lane], 1);
+      mbar_init(&ctl->v_full[lane], 2);
+      mbar_init(&ctl->v_empty[lane], 1);
+    } else if (lane < kStages + 2) {
+      const int i = lane - kStages;
       mbar_init(&ctl->s_full[i], 1);
       mbar_init(&ctl->s_free[i], 8);    // one arrival per warp: 4 warps of the warpgroup x 2 CTAs
       mbar_init(&ctl->pv_done[i], 1);
       mbar_init(&ctl->m_pub[i], 4);
+      mbar_init(&ctl->epi[i], 8);
+    } else if (lane == kStages + 2) {
+      mbar_init(&ctl->q_ready, 16);     // one arrival per softmax warp of both CTAs
+      mbar_init(&ctl->p_full, 8);
+      mbar_init(&ctl->o_done, 1);
+      mbar_init(&ctl->drain, 2);
+      mbar_init(&ctl->anc_ready, 1);
+      ctl->abort_flag = 0;
+    } else if (lane == kStages + 3) {
+      prefetch_tensormap(&maps.kp);
+      prefetch_tensormap(&maps.vp);
+      prefetch_tensormap(&maps.kt);
+      prefetch_tensormap(&maps.vt);
     }
-    mbar_init(&ctl->p_full, 8);
-    mbar_init(&ctl->o_done, 1);
-    mbar_init(&ctl->drain, 2);
-    mbar_init(&ctl->anc_ready, 1);
-    mbar_init(&ctl->epi[0], 8);
-    mbar_init(&ctl->epi[1], 8);
-    ctl->abort_flag = 0;
     fence_mbar_init();
-    prefetch_tensormap(&maps.kp);
-    prefetch_tensormap(&maps.vp);
-    prefetch_tensormap(&maps.kt);
-    prefetch_tensormap(&maps.vt);
+  } else if (warp == kMmaWarp) {
+    // tensor memory for the pair: both CTAs' warps with this index allocate all 512 columns
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                 "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   cluster_sync_all();                    // both CTAs' barriers exist before anyone signals them
   bool ok = true;
@@ -301,12 +309,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       }
     }
   } else {
-    if (warp == kMmaWarp) {
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
-                   "r"(512u)
-                   : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    } else if (warp == kTreeWarp) {
+    if (warp == kTreeWarp) {
       // registers first: the softmax warpgroups cannot grow until every warp of this warpgroup has shrunk
       setmaxnreg_dec<kRegsOther>();
       ctl->parent[lane] = lane < p.T ? a.parent[lane] : -1;
