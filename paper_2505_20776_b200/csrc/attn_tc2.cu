@@ -77,9 +77,17 @@ __device__ __forceinline__ uint32_t cluster_rank() {
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
   return r;
 }
-__device__ __forceinline__ void cluster_sync_all() {
+__device__ __forceinline__ void cluster_arrive() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Execution barrier only (no ordering of global memory): an arrival does not wait for the thread's
+// outstanding stores.
+__device__ __forceinline__ void cluster_sync_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
 }
 __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
   uint32_t r;
@@ -184,40 +192,11 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   const long long spx_t_start = clock64();
 #endif
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint32_t rank = cluster_rank();
-  const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
-  const int unit_lo = spx_unit_start(p, cl), unit_hi = spx_unit_start(p, cl + 1);
 
-  // The first segment's Q rows are requested before anything else, with asynchronous copies into a
-  // shared-memory scratch, so that their latency (a first touch of the page costs a TLB miss on top
-  // of DRAM) runs under the set-up instead of delaying the first S MMA.  8 lanes copy the 128 bytes
-  // a thread needs of one row (warpgroup 0: first 64 elements, warpgroup 1: the rest); 16-byte chunks
-  // are XOR-swizzled by the row so that the copies and the later per-row reads are conflict-free.
-  // The scratch (4 KB per warp) is the tail of the V ring, which the producer leaves alone until
-  // the first S MMA is done.
-  if (warp < kProducerWarp && unit_lo < unit_hi) {
-    const int prob = unit_lo / p.UPP;
-    const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
-    const int r0 = rblk * p.RB + (int)rank * 128 + (warp & 3) * 32;
-    const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + (warp >> 2) * 64;
-    unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int row = it * 4 + (lane >> 3), rw = r0 + row;
-      unsigned char* dst = scratch + row * 128 + (((lane & 7) ^ (row & 7)) << 4);
-      if (rw < p.rows) {
-        const __nv_bfloat16* src = qbase + (long long)(rw / p.G) * a.q_st + (long long)(rw % p.G) * a.q_sh + (lane & 7) * 8;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-      } else {
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  } else if (warp == kTreeWarp && lane == 0) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.parent));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.parent + 32));
-  }
-
+  // The cluster barrier that makes both CTAs' mbarriers visible is split: the producer warp
+  // initialises the barriers and arrives, every other warp arrives at once, and each warp waits just
+  // before it first touches a barrier.  What needs no barrier (the Q copies, the tensor-memory
+  // allocation, the ancestor masks) runs in between.
   if (warp == kProducerWarp) {
     // one barrier per lane (the four ring arrays first), so that the set-up is not 40 serial inits
     if (lane < kStages) {
@@ -239,26 +218,69 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       mbar_init(&ctl->drain, 2);
       mbar_init(&ctl->anc_ready, 1);
       ctl->abort_flag = 0;
-    } else if (lane == kStages + 3) {
-      prefetch_tensormap(&maps.kp);
-      prefetch_tensormap(&maps.vp);
-      prefetch_tensormap(&maps.kt);
-      prefetch_tensormap(&maps.vt);
     }
     fence_mbar_init();
-  } else if (warp == kMmaWarp) {
+  }
+  cluster_arrive();
+
+  const uint32_t rank = cluster_rank();
+  const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
+  const int unit_lo = spx_unit_start(p, cl), unit_hi = spx_unit_start(p, cl + 1);
+
+  // The first segment's Q rows are requested before anything else, with asynchronous copies into a
+  // shared-memory scratch, so that their latency (a first touch of the page costs a TLB miss on top
+  // of DRAM) runs under the set-up instead of delaying the first S MMA.  8 lanes copy the 128 bytes
+  // a thread needs of one row (warpgroup 0: first 64 elements, warpgroup 1: the rest); 16-byte chunks
+  // are XOR-swizzled by the row so that the copies and the later per-row reads are conflict-free.
+  // The scratch (4 KB per warp) is the tail of the V ring, which the producer leaves alone until
+  // the first S MMA is done.
+  if (warp < kProducerWarp && unit_lo < unit_hi) {
+    const int prob = unit_lo / p.UPP;
+    const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
+    const int r0 = rblk * p.RB + (int)rank * 128 + (warp & 3) * 32;
+    const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + (warp >> 2) * 64;
+    unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
+    int t_row = (r0 + (lane >> 3)) / p.G, i_row = (r0 + (lane >> 3)) - t_row * p.G;     // row = node * G + head
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+      const int row = it * 4 + (lane >> 3), rw = r0 + row;
+      unsigned char* dst = scratch + row * 128 + (((lane & 7) ^ (row & 7)) << 4);
+      if (it > 0) {
+        i_row += 4;
+        while (i_row >= p.G) {
+          i_row -= p.G;
+          ++t_row;
+        }
+      }
+      if (rw < p.rows) {
+        const __nv_bfloat16* src = qbase + (long long)t_row * a.q_st + (long long)i_row * a.q_sh + (lane & 7) * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+
+  if (warp == kProducerWarp && lane == 0) {
+    prefetch_tensormap(&maps.kp);
+    prefetch_tensormap(&maps.vp);
+    prefetch_tensormap(&maps.kt);
+    prefetch_tensormap(&maps.vt);
+  }
+  if (warp == kMmaWarp) {
     // tensor memory for the pair: both CTAs' warps with this index allocate all 512 columns
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
-  cluster_sync_all();                    // both CTAs' barriers exist before anyone signals them
   bool ok = true;
 
   if (warp == kProducerWarp) {
     // ================================ TMA producer (each CTA loads its halves) ===============
     setmaxnreg_dec<kRegsOther>();
+    cluster_wait();                        // both CTAs' barriers exist
     if (lane == 0) {
       uint32_t kp = 0, vp = 0;
       const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
@@ -333,11 +355,15 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         }
         ctl->anc[t] = m;
       }
+      cluster_wait();                      // this CTA's barriers exist
       warp_arrive(&ctl->anc_ready, lane);
     }
     // the tensor-memory base address is visible to everybody who uses it (not the producer, not the tree warp)
     tc_fence_before();
-    if (warp != kTreeWarp) named_bar_sync(1, kThreads - 64);
+    if (warp != kTreeWarp) {
+      named_bar_sync(1, kThreads - 64);
+      cluster_wait();                      // both CTAs' barriers exist
+    }
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
 
@@ -449,12 +475,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const int r = rblk * p.RB + rr;
         const bool valid = r < p.rows;
         const int t_node = valid ? r / p.G : 0;
-        if (seg == 0) {
-          ok = mbar_wait(&ctl->anc_ready, 0, abort_flag);
-          if (!ok) break;
-        }
-        const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
-
         // Q row of this thread -> tensor memory (warpgroup 0: first 64 elements, warpgroup 1: the rest)
         {
           uint32_t qv[32];
@@ -488,6 +508,11 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           tc_fence_before();
           warp_arrive_cluster(q_ready_l, lane);
         }
+        if (seg == 0) {
+          ok = mbar_wait(&ctl->anc_ready, 0, abort_flag);
+          if (!ok) break;
+        }
+        const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
 
         float m_loc = -INFINITY, l = 0.f;        // l is relative to m_loc
         for (int j = wg; j < n && ok; j += 2) {
@@ -693,10 +718,12 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           }
         }
         if (lane == 0) SPX_EVT2(2 + warp, 62);
-        warp_arrive(&ctl->epi[1], lane);                 // l_x and m_row may be reused
-        ok = mbar_wait(&ctl->epi[1], seg & 1, abort_flag);
-        ++seg;
         u += n;
+        if (u < unit_hi) {
+          warp_arrive(&ctl->epi[1], lane);               // l_x and m_row may be reused
+          ok = mbar_wait(&ctl->epi[1], seg & 1, abort_flag);
+        }
+        ++seg;
       }
     }
   }
@@ -704,8 +731,10 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
   tc_fence_before();
   if (tid == 0) SPX_EVT2(10, 0);
-  cluster_sync_all();
-  if (tid == 0) SPX_EVT2(10, 1);                    // the peer may still signal this CTA's barriers or read its halves
+  // The peer may still signal this CTA's barriers or read its halves, and tensor memory is freed by one
+  // warp for all: everybody meets once more.  The partial results written above need no ordering here.
+  cluster_sync_relaxed();
+  if (tid == 0) SPX_EVT2(10, 1);
   if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(ctl->tmem_base), "r"(512u) : "memory");
