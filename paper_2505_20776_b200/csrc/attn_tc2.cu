@@ -31,6 +31,7 @@ using namespace sm100;
 
 struct Tc2Maps {
   CUtensorMap kp, vp, kt, vt;
+  CUtensorMap q;      // Q as [T][Hq][128] with boxes of 64 x G x 128/G: the 128 stacked rows of one CTA
 };
 
 namespace {
@@ -62,6 +63,7 @@ struct Ctrl {
   uint64_t m_pub[2];            // this CTA: 4 arrivals, reference maxima of the tile are published
   uint64_t drain;
   uint64_t anc_ready;           // this CTA: the ancestor masks are in shared memory
+  uint64_t q_land;              // this CTA: the first segment's Q rows have landed in the scratch (TMA)
   uint64_t epi[2];              // this CTA: 8 arrivals, the two meeting points of a segment's epilogue
   unsigned long long anc[64];
   int parent[64];
@@ -217,6 +219,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       mbar_init(&ctl->o_done, 1);
       mbar_init(&ctl->drain, 2);
       mbar_init(&ctl->anc_ready, 1);
+      mbar_init(&ctl->q_land, 1);
       ctl->abort_flag = 0;
     }
     fence_mbar_init();
@@ -227,42 +230,26 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
   const int unit_lo = spx_unit_start(p, cl), unit_hi = spx_unit_start(p, cl + 1);
 
-  // The first segment's Q rows are requested before anything else, with asynchronous copies into a
-  // shared-memory scratch, so that their latency (a first touch of the page costs a TLB miss on top
-  // of DRAM) runs under the set-up instead of delaying the first S MMA.  8 lanes copy the 128 bytes
-  // a thread needs of one row (warpgroup 0: first 64 elements, warpgroup 1: the rest); 16-byte chunks
-  // are XOR-swizzled by the row so that the copies and the later per-row reads are conflict-free.
-  // The scratch (4 KB per warp) is the tail of the V ring, which the producer leaves alone until
-  // the first S MMA is done.
-  if (warp < kProducerWarp && unit_lo < unit_hi) {
+  // The first segment's Q rows are requested before anything else, into a shared-memory scratch, so
+  // that their latency runs under the set-up instead of delaying the first S MMA.  The scratch holds
+  // the CTA's 128 rows twice 64 elements (warpgroup 0 reads the first 64 elements of a row, warpgroup
+  // 1 the rest), 128 bytes per row with the 16-byte chunks XOR-swizzled by the row (the TMA 128-byte
+  // swizzle), so that the per-row reads are conflict-free.  It is the tail of the V ring, which the
+  // producer leaves alone until the first S MMA is done.  One thread fetches it with two TMA boxes
+  // of 64 elements x G heads x 128/G nodes: exactly the stacked rows (G is a power of two), rows
+  // past the tree zero-filled.
+  if (warp == kProducerWarp && lane == 0 && unit_lo < unit_hi) {
     const int prob = unit_lo / p.UPP;
     const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
-    const int r0 = rblk * p.RB + (int)rank * 128 + (warp & 3) * 32;
-    const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + (warp >> 2) * 64;
-    unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
-    int t_row = (r0 + (lane >> 3)) / p.G, i_row = (r0 + (lane >> 3)) - t_row * p.G;     // row = node * G + head
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-      const int row = it * 4 + (lane >> 3), rw = r0 + row;
-      unsigned char* dst = scratch + row * 128 + (((lane & 7) ^ (row & 7)) << 4);
-      if (it > 0) {
-        i_row += 4;
-        while (i_row >= p.G) {
-          i_row -= p.G;
-          ++t_row;
-        }
-      }
-      if (rw < p.rows) {
-        const __nv_bfloat16* src = qbase + (long long)t_row * a.q_st + (long long)i_row * a.q_sh + (lane & 7) * 8;
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-      } else {
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
+    const int t0 = (rblk * p.RB + (int)rank * 128) / p.G;
+    unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes;
+    mbar_arrive_expect_tx(&ctl->q_land, 2 * kStageBytes);
+    tma_load_3d(scratch, &maps.q, &ctl->q_land, 0, g * p.G, t0);
+    tma_load_3d(scratch + kStageBytes, &maps.q, &ctl->q_land, 64, g * p.G, t0);
   }
 
   if (warp == kProducerWarp && lane == 0) {
+    prefetch_tensormap(&maps.q);
     prefetch_tensormap(&maps.kp);
     prefetch_tensormap(&maps.vp);
     prefetch_tensormap(&maps.kt);
@@ -284,50 +271,71 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     if (lane == 0) {
       uint32_t kp = 0, vp = 0;
       const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
-
       const uint32_t vfull0 = map_to_cta(smem_u32(&ctl->v_full[0]), 0);
-      for (int u = unit_lo; u < unit_hi && ok;) {
-        const int prob = u / p.UPP;
-        const int tile_lo = u - prob * p.UPP;
-        const int n = min(p.UPP - tile_lo, unit_hi - u);
-        const int g = prob / p.n_rblk;
-        for (int j = 0; j < n && ok; ++j) {
-          const int tile = tile_lo + j;
-          const bool is_tree = tile == p.TPH;
-          // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A
-          // full ring requested at once by every SM sits in the memory system's queues in no
-          // particular order, and tile 0 would arrive last as often as first.
-          if (kp == 2) {
-            ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
-            if (!ok) break;
-          }
-          {   // K half: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
-            const int stage = kp % kStages;
-            ok = wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            const uint32_t bar = kfull0 + stage * 8;
-            const uint32_t dst = smem_u32(ring + stage * kStageBytes);
-            const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
-            const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
-            arrive_expect_tx_cluster(bar, kStageBytes);
-            tma_load_3d_pair(dst, m, bar, 0, g, key0);
-            tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
-            SPX_EVT2(0, 2 * j);
-            ++kp;
-          }
-          {   // V half: value columns [64*rank, 64*rank+64) of all 128 keys
-            const int stage = vp % kStages;
-            ok = wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            const uint32_t bar = vfull0 + stage * 8;
-            const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
-            arrive_expect_tx_cluster(bar, kStageBytes);
-            tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
-            SPX_EVT2(0, 2 * j + 1);
-            ++vp;
-          }
+      // position in the line of units
+      struct Cursor {
+        int unit, tile, prob, g;
+      };
+      auto step = [&](Cursor& c) {
+        ++c.unit;
+        if (++c.tile == p.UPP) {
+          c.tile = 0;
+          ++c.prob;
+          c.g = c.prob / p.n_rblk;
         }
-        u += n;
+      };
+      // K half of a unit: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
+      auto load_k = [&](const Cursor& c) -> bool {
+        const int tile = c.tile, g = c.g;
+        const bool is_tree = tile == p.TPH;
+        const int stage = kp % kStages;
+        if (!wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag)) return false;
+        const uint32_t bar = kfull0 + stage * 8;
+        const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+        const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
+        const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
+        arrive_expect_tx_cluster(bar, kStageBytes);
+        tma_load_3d_pair(dst, m, bar, 0, g, key0);
+        tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
+        SPX_EVT2(0, 2 * (int)kp);
+        ++kp;
+        return true;
+      };
+      // V half of a unit: value columns [64*rank, 64*rank+64) of all 128 keys
+      auto load_v = [&](const Cursor& c) -> bool {
+        const int tile = c.tile, g = c.g;
+        const bool is_tree = tile == p.TPH;
+        const int stage = vp % kStages;
+        if (!wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag)) return false;
+        const uint32_t bar = vfull0 + stage * 8;
+        const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
+        arrive_expect_tx_cluster(bar, kStageBytes);
+        tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
+        SPX_EVT2(0, 2 * (int)vp + 1);
+        ++vp;
+        return true;
+      };
+      // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A full
+      // ring requested at once by every SM sits in the memory system's queues in no particular order,
+      // and tile 0 would arrive last as often as first.
+      Cursor ck;
+      ck.unit = unit_lo;
+      ck.prob = unit_lo / p.UPP;
+      ck.tile = unit_lo - ck.prob * p.UPP;
+      ck.g = ck.prob / p.n_rblk;
+      Cursor cv = ck;
+      for (int i = 0; i < 2 && ck.unit < unit_hi && ok; ++i) {
+        ok = load_k(ck);
+        step(ck);
+        if (ok) ok = load_v(cv);
+        step(cv);
+      }
+      if (ok && unit_lo < unit_hi) ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
+      while (ok && ck.unit < unit_hi) {
+        ok = load_k(ck);
+        step(ck);
+        if (ok) ok = load_v(cv);
+        step(cv);
       }
     }
   } else {
@@ -482,8 +490,8 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           if (seg == 0) {
             // requested at kernel start (see above)
             const unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncwarp();
+            ok = mbar_wait(&ctl->q_land, 0, abort_flag);
+            if (!ok) break;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               const uint4 y = *reinterpret_cast<const uint4*>(scratch + lane * 128 + ((j ^ (lane & 7)) << 4));
@@ -771,6 +779,19 @@ bool encode_map2(CUtensorMap* m, const void* ptr, long long n1, long long s1, lo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Q [T][Hq][128] (element strides q_st, q_sh, 1) with boxes of 64 elements x G heads x 128/G nodes.
+bool encode_q_map(CUtensorMap* m, const void* ptr, int T, int Hq, int G, long long q_st, long long q_sh) {
+  EncodeTiledFn fn = encode_fn2();
+  if (!fn || G > 128 || 128 % G != 0) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)T};
+  const cuuint64_t strides[2] = {(cuuint64_t)q_sh * 2, (cuuint64_t)q_st * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)G, (cuuint32_t)(128 / G)};
+  const cuuint32_t es[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <bool SCORE>
 cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
   static bool configured = false;
@@ -810,6 +831,7 @@ cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launc
     maps.kp = maps.kt;
     maps.vp = maps.vt;
   }
+  ok = ok && encode_q_map(&maps.q, a.Q, p.T, p.Hq, p.G, a.q_st, a.q_sh);
   if (!ok) return cudaErrorInvalidValue;
   const cudaError_t e = p.want_score ? launch2<true>(a, maps, st) : launch2<false>(a, maps, st);
   *n_launches += 1;
