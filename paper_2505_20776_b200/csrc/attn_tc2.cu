@@ -622,6 +622,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           }
 
           const float neg_m = -m_new;
+          const uint64_t scale2x2 = pack_f32x2(scale2, scale2), neg_mx2 = pack_f32x2(neg_m, neg_m);
           const bool score = SCORE && !is_tree;
           float* mass = nullptr;
           if (score) {
@@ -632,17 +633,27 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           float csum = 0.f;
           uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
           auto exp_chunk = [&](uint32_t (&v)[32], uint32_t (&pk)[16], int c) {
-#pragma unroll
-            for (int k = 0; k < 32; ++k)
-              v[k] = __float_as_uint(ex2_approx(fmaf(__uint_as_float(v[k]), scale2, neg_m)));
-            float gs0 = 0.f, gs1 = 0.f, gs2 = 0.f, gs3 = 0.f;
+            // two elements per fma and per add (packed fp32 pairs); the exponential itself is per element
+            uint64_t acc01 = 0ull, acc23 = 0ull;
 #pragma unroll
             for (int k = 0; k < 32; k += 4) {
-              gs0 += __uint_as_float(v[k]);
-              gs1 += __uint_as_float(v[k + 1]);
-              gs2 += __uint_as_float(v[k + 2]);
-              gs3 += __uint_as_float(v[k + 3]);
+              float e0, e1, e2, e3;
+              unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), scale2x2, neg_mx2), e0, e1);
+              unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3])), scale2x2, neg_mx2), e2, e3);
+              e0 = ex2_approx(e0);
+              e1 = ex2_approx(e1);
+              e2 = ex2_approx(e2);
+              e3 = ex2_approx(e3);
+              acc01 = add_f32x2(acc01, pack_f32x2(e0, e1));
+              acc23 = add_f32x2(acc23, pack_f32x2(e2, e3));
+              v[k] = __float_as_uint(e0);
+              v[k + 1] = __float_as_uint(e1);
+              v[k + 2] = __float_as_uint(e2);
+              v[k + 3] = __float_as_uint(e3);
             }
+            float gs0, gs1, gs2, gs3;
+            unpack_f32x2(acc01, gs0, gs1);
+            unpack_f32x2(acc23, gs2, gs3);
             const float gs = (gs0 + gs1) + (gs2 + gs3);
             l += gs;
             if (score) {
