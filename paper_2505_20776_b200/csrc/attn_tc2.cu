@@ -225,6 +225,10 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     fence_mbar_init();
   }
   cluster_arrive();
+  // The kernel after this one (the merge) may be set up while this one runs; this one touches global
+  // memory only once the kernel before it has completed (its set-up so far has used none).
+  pdl_launch_dependents();
+  if (warp != kMmaWarp) pdl_wait();
 
   const uint32_t rank = cluster_rank();
   const int cl = blockIdx.x >> 1;                        // the plan's "CTA" index is the cluster index
@@ -261,6 +265,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
                  "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    pdl_wait();
   }
   bool ok = true;
 
@@ -816,13 +821,15 @@ cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, attn_tc2_kernel<SCORE>, a, maps);
 }
 

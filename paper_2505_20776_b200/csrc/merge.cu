@@ -8,10 +8,12 @@
 // exponential sum rescaled from its tile's reference maximum to the row's final lse, i.e. the
 // exactly normalised probability mass, and divides by Hq.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace {
 
 constexpr float kLn2 = 0.693147180559945309417f;
+constexpr int kMergeSmemCap = 100 * 1024;          // bytes of dynamic shared memory requested only to limit residency
 constexpr float kLog2e = 1.44269504088896340736f;
 
 // Block = 8 warps; warp w handles one 16-byte column group d4 for 32 consecutive rows of one
@@ -19,6 +21,8 @@ constexpr float kLog2e = 1.44269504088896340736f;
 // independent of each other.
 __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
+  sm100::pdl_launch_dependents();
+  sm100::pdl_wait();                               // the partial results of the attention kernel are complete
   const int blocks_per_prob = p.RB / 32;
   const int prob = blockIdx.x / blocks_per_prob;
   const int rr0 = (blockIdx.x - prob * blocks_per_prob) * 32;
@@ -107,9 +111,28 @@ __global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ Attn
 cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches) {
   const AttnPlan& p = a.plan;
   const dim3 grid(p.NP * (p.RB / 32), p.D / 32);
-  merge_kernel<<<grid, 256, 0, st>>>(a);
+  // Launched so that its blocks may be resident (waiting) before the attention kernel has finished.
+  // Blocks become resident wherever an SM has room, so without a limit the SMs that the attention
+  // kernel leaves first would take eight blocks each and a quarter of the SMs would do all the work:
+  // an (unused) dynamic shared-memory request caps residency at two blocks per SM.
+  static bool configured = false;
+  if (!configured) {
+    const cudaError_t ec = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemCap);
+    if (ec != cudaSuccess) return ec;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = kMergeSmemCap;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, merge_kernel, a);
   *n_launches += 1;
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (p.want_score && p.NC > 0) {
     const dim3 sgrid((p.NC + 255) / 256, p.T);

@@ -232,6 +232,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may
+// start while the kernel before it in the stream still runs: pdl_wait() returns once that kernel
+// has completed and its writes are visible (at once if the launch was an ordinary one);
+// pdl_launch_dependents() lets the kernel after this one start its own prologue early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Packed pairs of fp32 (sm_100 has two-wide fp32 fma/add): one instruction for two elements.
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
   uint64_t r;
