@@ -16,9 +16,49 @@ constexpr float kLn2 = 0.693147180559945309417f;
 constexpr int kMergeSmemCap = 100 * 1024;          // bytes of dynamic shared memory requested only to limit residency
 constexpr float kLog2e = 1.44269504088896340736f;
 
-// Block = 8 warps; warp w handles one 16-byte column group d4 for 32 consecutive rows of one
-// problem, so every partial read is a 512-byte coalesced segment and all reads of a thread are
-// independent of each other.
+// Block = 8 warps; warp w handles two 16-byte column groups (d4, d4 + 1) for 32 consecutive rows of
+// one problem, so every partial read is a 512-byte coalesced segment, all reads of a thread are
+// independent of each other, and the segment weights are computed once for eight output columns.
+template <int B>
+__device__ __forceinline__ void merge_batch(const float* __restrict__ pm, const float* __restrict__ pl,
+                                            const float* __restrict__ po, long long ostride, int RB, int s, int n,
+                                            float& M, float& Z, float4& acc0, float4& acc1) {
+  // Segments s .. s+n-1 (n <= B).  Every load of the batch is in flight at once: issued one by one
+  // they would each pay the full latency, and a second batch pays it a second time.
+  float ms[B], ls[B];
+  float4 v0[B], v1[B];
+#pragma unroll
+  for (int k = 0; k < B; ++k) {
+    const bool in = k < n;
+    const float4* q = reinterpret_cast<const float4*>(po + (s + k) * ostride);
+    ms[k] = in ? __ldcg(pm + (long long)(s + k) * RB) : -INFINITY;
+    ls[k] = in ? __ldcg(pl + (long long)(s + k) * RB) : 0.f;
+    v0[k] = in ? __ldcg(q) : make_float4(0.f, 0.f, 0.f, 0.f);
+    v1[k] = in ? __ldcg(q + RB) : make_float4(0.f, 0.f, 0.f, 0.f);     // next column group: RB float4 further on
+  }
+  float Mb = M;
+#pragma unroll
+  for (int k = 0; k < B; ++k) Mb = fmaxf(Mb, ms[k]);
+  const float carry = sm100::ex2_approx(M - Mb);    // 0 on the first batch (M = -inf)
+  Z *= carry;
+  acc0.x *= carry; acc0.y *= carry; acc0.z *= carry; acc0.w *= carry;
+  acc1.x *= carry; acc1.y *= carry; acc1.z *= carry; acc1.w *= carry;
+  M = Mb;
+#pragma unroll
+  for (int k = 0; k < B; ++k) {
+    const float w = sm100::ex2_approx(ms[k] - M);
+    Z = fmaf(ls[k], w, Z);
+    acc0.x = fmaf(w, v0[k].x, acc0.x);
+    acc0.y = fmaf(w, v0[k].y, acc0.y);
+    acc0.z = fmaf(w, v0[k].z, acc0.z);
+    acc0.w = fmaf(w, v0[k].w, acc0.w);
+    acc1.x = fmaf(w, v1[k].x, acc1.x);
+    acc1.y = fmaf(w, v1[k].y, acc1.y);
+    acc1.z = fmaf(w, v1[k].z, acc1.z);
+    acc1.w = fmaf(w, v1[k].w, acc1.w);
+  }
+}
+
 __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
   sm100::pdl_launch_dependents();
@@ -32,58 +72,41 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   const int rr = rr0 + lane;
   const int r = rblk * p.RB + rr;
   if (r >= p.rows) return;
-  const int c_first = spx_unit_owner(p, prob * p.UPP);
-  const int c_last = spx_unit_owner(p, (prob + 1) * p.UPP - 1);
+  int c_first, c_last;
+  if (p.cpp > 0 && p.UPP >= p.cpp) {               // every one of the problem's cpp workers has a segment
+    c_first = prob * p.cpp;
+    c_last = c_first + p.cpp - 1;
+  } else {
+    c_first = spx_unit_owner(p, prob * p.UPP);
+    c_last = spx_unit_owner(p, (prob + 1) * p.UPP - 1);
+  }
   const int nseg = c_last - c_first + 1;
   const int slot0 = c_first + prob;
   const int nd4 = p.D / 4;
-  const int d4 = blockIdx.y * 8 + warp;
+  const int d4 = (blockIdx.y * 8 + warp) * 2;
 
   const float* pm = a.ws + p.off_part_m + (long long)slot0 * p.RB + rr;
   const float* pl = a.ws + p.off_part_l + (long long)slot0 * p.RB + rr;
   const float* po = a.ws + p.off_part_o + (((long long)slot0 * nd4 + d4) * p.RB + rr) * 4;
   const long long ostride = (long long)nd4 * p.RB * 4;
 
-  // Batches of 8 segments with every load of a batch in flight at once (the loads of one thread are
-  // independent; issued one by one they would each pay the full memory latency).
   float M = -INFINITY, Z = 0.f;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < nseg; s += 8) {
-    float ms[8], ls[8];
-    float4 v[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const bool in = s + k < nseg;
-      ms[k] = in ? __ldcg(pm + (long long)(s + k) * p.RB) : -INFINITY;
-      ls[k] = in ? __ldcg(pl + (long long)(s + k) * p.RB) : 0.f;
-      v[k] = in ? __ldcg(reinterpret_cast<const float4*>(po + (s + k) * ostride)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    float Mb = M;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) Mb = fmaxf(Mb, ms[k]);
-    const float carry = exp2f(M - Mb);              // 0 on the first batch (M = -inf)
-    Z *= carry;
-    acc.x *= carry; acc.y *= carry; acc.z *= carry; acc.w *= carry;
-    M = Mb;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const float w = exp2f(ms[k] - M);
-      Z = fmaf(ls[k], w, Z);
-      acc.x = fmaf(w, v[k].x, acc.x);
-      acc.y = fmaf(w, v[k].y, acc.y);
-      acc.z = fmaf(w, v[k].z, acc.z);
-      acc.w = fmaf(w, v[k].w, acc.w);
-    }
-  }
+  float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
+  for (int s = 0; s < nseg; s += 12) merge_batch<12>(pm, pl, po, ostride, p.RB, s, min(12, nseg - s), M, Z, acc0, acc1);
+
   const float inv = 1.f / Z;
   const int t = r / p.G, h = g * p.G + r % p.G;
   if (d4 == 0) a.lse[(long long)h * p.T + t] = (M + log2f(Z)) * kLn2;
-  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-  __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-  uint2 pk;
-  pk.x = *reinterpret_cast<uint32_t*>(&lo);
-  pk.y = *reinterpret_cast<uint32_t*>(&hi);
-  *reinterpret_cast<uint2*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
+  __nv_bfloat162 b0 = __floats2bfloat162_rn(acc0.x * inv, acc0.y * inv);
+  __nv_bfloat162 b1 = __floats2bfloat162_rn(acc0.z * inv, acc0.w * inv);
+  __nv_bfloat162 b2 = __floats2bfloat162_rn(acc1.x * inv, acc1.y * inv);
+  __nv_bfloat162 b3 = __floats2bfloat162_rn(acc1.z * inv, acc1.w * inv);
+  uint4 pk;
+  pk.x = *reinterpret_cast<uint32_t*>(&b0);
+  pk.y = *reinterpret_cast<uint32_t*>(&b1);
+  pk.z = *reinterpret_cast<uint32_t*>(&b2);
+  pk.w = *reinterpret_cast<uint32_t*>(&b3);
+  *reinterpret_cast<uint4*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
 }
 
 __global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ AttnArgs a) {
@@ -110,7 +133,7 @@ __global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ Attn
 
 cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches) {
   const AttnPlan& p = a.plan;
-  const dim3 grid(p.NP * (p.RB / 32), p.D / 32);
+  const dim3 grid(p.NP * (p.RB / 32), p.D / 64);
   // Launched so that its blocks may be resident (waiting) before the attention kernel has finished.
   // Blocks become resident wherever an SM has room, so without a limit the SMs that the attention
   // kernel leaves first would take eight blocks each and a quarter of the SMs would do all the work:
