@@ -636,6 +636,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             a.ws[p.off_mref + rowbase] = m_new;
           }
           float csum = 0.f;
+          float cg[4] = {0.f, 0.f, 0.f, 0.f};      // chunk size 32: the tile's four chunk sums, stored as one float4
           uint32_t pk0[16], pk1[16], pk2[16], pk3[16];
           auto exp_chunk = [&](uint32_t (&v)[32], uint32_t (&pk)[16], int c) {
             // two elements per fma and per add (packed fp32 pairs); the exponential itself is per element
@@ -662,7 +663,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             const float gs = (gs0 + gs1) + (gs2 + gs3);
             l += gs;
             if (score) {
-              if (p.C >= 32) {
+              if (p.C == 32) {
+                cg[c] = gs;
+              } else if (p.C > 32) {
                 csum += gs;
                 if ((((c + 1) * 32) & (p.C - 1)) == 0) {
                   mass[((c + 1) * 32) / p.C - 1] = csum;
@@ -687,6 +690,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           exp_chunk(s1, pk1, 1);
           exp_chunk(s2, pk2, 2);
           exp_chunk(s3, pk3, 3);
+          if (score && p.C == 32) *reinterpret_cast<float4*>(mass) = make_float4(cg[0], cg[1], cg[2], cg[3]);
           // the P buffer is shared by all tiles: the PV of the previous tile must have read it
           ok = wait_prev_pv();
           if (!ok) break;

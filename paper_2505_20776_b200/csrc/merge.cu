@@ -4,9 +4,9 @@
 // merge_kernel: for each query row: M = max_s m_s,
 // Z = sum_s l_s 2^(m_s - M), lse = (M + log2 Z) ln 2, O = sum_s O~_s 2^(m_s - M) / Z.
 //
-// score_kernel: one thread per (tree node, chunk): sums over all query heads the chunk's
-// exponential sum rescaled from its tile's reference maximum to the row's final lse, i.e. the
-// exactly normalised probability mass, and divides by Hq.
+// score_kernel: for every (tree node, chunk) sums over all query heads the chunk's exponential sum
+// rescaled from its tile's reference maximum to the row's final lse, i.e. the exactly normalised
+// probability mass, and divides by Hq.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -109,24 +109,46 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   *reinterpret_cast<uint4*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
 }
 
-__global__ void __launch_bounds__(256) score_kernel(const __grid_constant__ AttnArgs a) {
+// One thread per (tree node t, key tile, group of VW chunks of the tile): consecutive threads are
+// consecutive nodes, whose G stacked rows lie next to each other in the per-row arrays, so a warp
+// reads whole lines; the VW chunk sums of a row are one vector load.
+template <int VW>
+__global__ void __launch_bounds__(64) score_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
-  const int t = blockIdx.y;
-  const int c = blockIdx.x * 256 + threadIdx.x;
-  if (c >= p.NC) return;
-  const int tile = c / p.CPT, cc = c - tile * p.CPT;
-  float acc = 0.f;
-  for (int h = 0; h < p.Hq; ++h) {
-    const int g = h / p.G, i = h - g * p.G;
-    const int r = t * p.G + i;
-    const int rblk = r / p.RB, rr = r - rblk * p.RB;
-    const int prob = g * p.n_rblk + rblk;
-    const long long base = ((long long)prob * p.TPH + tile) * p.RB + rr;
-    const float lse2 = a.lse[(long long)h * p.T + t] * kLog2e;
-    const float f = exp2f(a.ws[p.off_mref + base] - lse2);
-    acc = fmaf(a.ws[p.off_mass + base * p.CPT + cc], f, acc);
+  const int t = threadIdx.x;
+  const int tile = blockIdx.x;
+  const int c0 = blockIdx.y * VW;                  // first chunk of the group inside the tile
+  if (t >= p.T) return;
+  float acc[VW];
+#pragma unroll
+  for (int k = 0; k < VW; ++k) acc[k] = 0.f;
+  for (int g = 0; g < p.Hkv; ++g) {
+    for (int i = 0; i < p.G; ++i) {
+      const int r = t * p.G + i;
+      const int rblk = r / p.RB, rr = r - rblk * p.RB;
+      const int prob = g * p.n_rblk + rblk;
+      const long long base = ((long long)prob * p.TPH + tile) * p.RB + rr;
+      const float lse2 = a.lse[(long long)(g * p.G + i) * p.T + t] * kLog2e;
+      const float f = exp2f(a.ws[p.off_mref + base] - lse2);
+      const float* m = a.ws + p.off_mass + base * p.CPT + c0;
+      if (VW == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(m);
+        acc[0] = fmaf(v.x, f, acc[0]);
+        acc[1 % VW] = fmaf(v.y, f, acc[1 % VW]);
+        acc[2 % VW] = fmaf(v.z, f, acc[2 % VW]);
+        acc[3 % VW] = fmaf(v.w, f, acc[3 % VW]);
+      } else {
+#pragma unroll
+        for (int k = 0; k < VW; ++k) acc[k] = fmaf(m[k], f, acc[k]);
+      }
+    }
   }
-  a.chunk_score[(long long)t * p.NC + c] = acc / (float)p.Hq;
+  const float inv = 1.f / (float)p.Hq;
+#pragma unroll
+  for (int k = 0; k < VW; ++k) {
+    const int c = tile * p.CPT + c0 + k;
+    if (c < p.NC) a.chunk_score[(long long)t * p.NC + c] = acc[k] * inv;
+  }
 }
 
 }  // namespace
@@ -158,8 +180,13 @@ cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches
   *n_launches += 1;
   if (e != cudaSuccess) return e;
   if (p.want_score && p.NC > 0) {
-    const dim3 sgrid((p.NC + 255) / 256, p.T);
-    score_kernel<<<sgrid, 256, 0, st>>>(a);
+    if (p.CPT >= 4) {
+      score_kernel<4><<<dim3(p.TPH, p.CPT / 4), 64, 0, st>>>(a);
+    } else if (p.CPT == 2) {
+      score_kernel<2><<<dim3(p.TPH, 1), 64, 0, st>>>(a);
+    } else {
+      score_kernel<1><<<dim3(p.TPH, 1), 64, 0, st>>>(a);
+    }
     *n_launches += 1;
     e = cudaGetLastError();
   }
