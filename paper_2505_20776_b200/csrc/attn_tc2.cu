@@ -150,6 +150,12 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// Asks for a tile to be brought into L2; needs no barrier and no shared memory.
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
 // D[tmem, both CTAs] (+)= A[tmem, own rows of each CTA] * B[smem halves of both CTAs]
 __device__ __forceinline__ void mma_ts_pair(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -250,6 +256,15 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     mbar_arrive_expect_tx(&ctl->q_land, 2 * kStageBytes);
     tma_load_3d(scratch, &maps.q, &ctl->q_land, 0, g * p.G, t0);
     tma_load_3d(scratch + kStageBytes, &maps.q, &ctl->q_land, 64, g * p.G, t0);
+    // The first K/V tiles can only be loaded once the pair's barriers are known to exist (a cluster
+    // barrier away); until then their halves are at least pulled into L2.
+    const int tile = unit_lo - prob * p.UPP;
+    const bool is_tree = tile == p.TPH;
+    const int key0 = is_tree ? 0 : tile * SPX_TILE_KEYS;
+    const CUtensorMap* mk = is_tree ? &maps.kt : &maps.kp;
+    tma_prefetch_3d(mk, 0, g, key0 + 64 * rank);
+    tma_prefetch_3d(mk, 64, g, key0 + 64 * rank);
+    tma_prefetch_3d(is_tree ? &maps.vt : &maps.vp, 64 * rank, g, key0);
   }
 
   if (warp == kProducerWarp && lane == 0) {
