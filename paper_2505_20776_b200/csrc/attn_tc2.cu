@@ -752,10 +752,10 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             for (int q4 = 0; q4 < 8; ++q4) {
               const float4 x = make_float4(__uint_as_float(v[q4 * 4]), __uint_as_float(v[q4 * 4 + 1]),
                                            __uint_as_float(v[q4 * 4 + 2]), __uint_as_float(v[q4 * 4 + 3]));
-              *reinterpret_cast<float4*>(po + ((long long)(wg * 16 + c * 8 + q4) * p.RB + rr) * 4) = x;
+              if (valid) *reinterpret_cast<float4*>(po + ((long long)(wg * 16 + c * 8 + q4) * p.RB + rr) * 4) = x;
             }
           }
-          if (wg == 0) {
+          if (wg == 0 && valid) {                        // rows past the last stacked row are never read
             a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_fin;
             a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l + ctl->l_x[row_t];
           }

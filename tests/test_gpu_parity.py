@@ -414,3 +414,47 @@ def test_paired_kernel_with_more_problems_than_clusters(cuda_device):
     w = _small(160, 80, 128, 96, 64, 32)          # rows = 128 -> one-CTA kernel, one short tile, many problems
     hp = make_hp(w, cuda_device)
     check_attn(hp, synth.make_layer(w), synth.make_tree(w), 96, 32)
+
+
+def test_back_to_back_calls_in_a_graph_share_a_workspace(cuda_device):
+    """Four calls with different inputs, one workspace, captured in one CUDA graph and replayed.
+
+    The attention and merge kernels are launched so that a kernel's set-up may overlap the tail of the
+    kernel before it; every call must still see the workspace only after the previous call is done with it.
+    """
+    w = synth.WORKLOADS["c1"]
+    dev = cuda_device
+    parent = synth.make_tree(w)
+    par = torch.from_numpy(parent).to(dev)
+    layers_cpu = [synth.make_layer(w, layer=i) for i in range(4)]
+    layers = [to_dev(t, dev) for t in layers_cpu]
+    T, Hq, D = w.n_tree, w.n_q_heads, w.head_dim
+    outs = [torch.zeros(T, Hq, D, dtype=torch.bfloat16, device=dev) for _ in layers]
+    lses = [torch.zeros(Hq, T, dtype=torch.float32, device=dev) for _ in layers]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    d = api.make_attn_desc(layers[0]["Q"], layers[0]["K_prefix"], layers[0]["K_tree"], outs[0], w.prefix_len,
+                           w.chunk_size)
+    ws = torch.zeros(api.specext_verify_attn_workspace(d), dtype=torch.uint8, device=dev)
+
+    def run():
+        for t, O, lse in zip(layers, outs, lses):
+            api.specext_verify_attn(d, t["Q"], t["K_prefix"], t["V_prefix"], t["K_tree"], t["V_tree"], par, O, lse,
+                                    None, ws, status)
+
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        run()
+        s.synchronize()
+        with torch.cuda.graph(g, stream=s):
+            run()
+        for O in outs:
+            O.zero_()
+        for _ in range(3):
+            g.replay()
+        s.synchronize()
+    assert int(status.item()) == 0
+    for t_cpu, O, lse in zip(layers_cpu, outs, lses):
+        O_ref, lse_ref, _ = oracle_layer(t_cpu, parent, w.prefix_len, w.chunk_size, None)
+        assert np.abs(f64(O) - O_ref).max() <= O_ATOL
+        assert np.abs(f64(lse) - lse_ref).max() <= LSE_ATOL
