@@ -285,6 +285,41 @@ def main():
         barrier()
         attn_us_mean = a.elapsed_time(b) * 1e3 / (rsteps * (NL - 1))
 
+        # ---- the other parts, each timed alone the same way (reported, not part of `value`) --
+        def timed_us(fn, calls):
+            fn()
+            stream.synchronize()
+            runner = fn
+            if not args.no_graph:
+                gg = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(gg, stream=stream):
+                    fn()
+                runner = gg.replay
+            runner()
+            barrier()
+            x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            x.record(stream)
+            for _ in range(rsteps):
+                runner()
+            y.record(stream)
+            barrier()
+            return x.elapsed_time(y) * 1e3 / (rsteps * calls)
+
+        n_sc = min(NL, 8)                                # 8 distinct layers = 0.5 GB of K/V: from HBM
+
+        def score_layers():
+            for i in range(n_sc):
+                hp.verify_attn(layers[i], parent, L, True)
+
+        def retrieval():
+            hp.select_chunks(row, L)
+            hp.gather_kv(dK, dV, L)
+
+        parts = {"scoreless_layer_us": attn_us_mean, "score_layer_us": timed_us(score_layers, n_sc),
+                 "select_gather_us": timed_us(retrieval, 1),
+                 "note": "each part replayed alone; select+gather re-reads the same 8 MB (L2-resident)"}
+        hp.verify_attn(layers[NL - 1], parent, L, True)  # leave the scores of the last layer in place
+
         # ---- end to end: host buffers, copies inside the timed region ----------------------
         e2e = None
         if args.e2e_steps > 0:
@@ -370,7 +405,7 @@ def main():
                            "cuda_graph": graph is not None, "replicas": world,
                            **({"profiling_layers": NL} if args.layers > 0 else {})},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-                "roofline": roof}
+                "roofline": roof, "parts": parts}
         if world == 1 and not args.no_cpu_baseline:
             ta, tr = oracle_sample(w, parent_np, 3)
             cpu_us = (sum(ta) / len(ta) + sum(tr) / len(tr) / NL) * 1e6

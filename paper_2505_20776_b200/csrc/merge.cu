@@ -109,46 +109,77 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   *reinterpret_cast<uint4*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
 }
 
-// One thread per (tree node t, key tile, group of VW chunks of the tile): consecutive threads are
-// consecutive nodes, whose G stacked rows lie next to each other in the per-row arrays, so a warp
-// reads whole lines; the VW chunk sums of a row are one vector load.
+// Block = 64 tree nodes x kScoreSlices slices of the KV heads, for one key tile and one group of VW
+// chunks of the tile.  Consecutive threads are consecutive nodes, whose G stacked rows lie next to
+// each other in the per-row arrays, so a warp reads whole lines; the VW chunk sums of a row are one
+// vector load.  A slice sums its KV heads in a fixed order and the slices are added in a fixed
+// order, so the result does not depend on the run.
+constexpr int kScoreSlices = 8;
+
 template <int VW>
-__global__ void __launch_bounds__(64) score_kernel(const __grid_constant__ AttnArgs a) {
+__global__ void __launch_bounds__(64 * kScoreSlices) score_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
-  const int t = threadIdx.x;
+  __shared__ float part[kScoreSlices][64][VW];
+  sm100::pdl_launch_dependents();
+  sm100::pdl_wait();                               // lse and the chunk sums are complete
+  const int t = threadIdx.x, slice = threadIdx.y;
   const int tile = blockIdx.x;
   const int c0 = blockIdx.y * VW;                  // first chunk of the group inside the tile
-  if (t >= p.T) return;
   float acc[VW];
 #pragma unroll
   for (int k = 0; k < VW; ++k) acc[k] = 0.f;
-  for (int g = 0; g < p.Hkv; ++g) {
-    for (int i = 0; i < p.G; ++i) {
-      const int r = t * p.G + i;
-      const int rblk = r / p.RB, rr = r - rblk * p.RB;
-      const int prob = g * p.n_rblk + rblk;
-      const long long base = ((long long)prob * p.TPH + tile) * p.RB + rr;
-      const float lse2 = a.lse[(long long)(g * p.G + i) * p.T + t] * kLog2e;
-      const float f = exp2f(a.ws[p.off_mref + base] - lse2);
-      const float* m = a.ws + p.off_mass + base * p.CPT + c0;
-      if (VW == 4) {
-        const float4 v = *reinterpret_cast<const float4*>(m);
-        acc[0] = fmaf(v.x, f, acc[0]);
-        acc[1 % VW] = fmaf(v.y, f, acc[1 % VW]);
-        acc[2 % VW] = fmaf(v.z, f, acc[2 % VW]);
-        acc[3 % VW] = fmaf(v.w, f, acc[3 % VW]);
-      } else {
+  if (t < p.T) {
+    for (int g = slice; g < p.Hkv; g += kScoreSlices) {
+      for (int i = 0; i < p.G; ++i) {
+        const int r = t * p.G + i;
+        const int rblk = r / p.RB, rr = r - rblk * p.RB;
+        const int prob = g * p.n_rblk + rblk;
+        const long long base = ((long long)prob * p.TPH + tile) * p.RB + rr;
+        const float lse2 = a.lse[(long long)(g * p.G + i) * p.T + t] * kLog2e;
+        const float f = exp2f(a.ws[p.off_mref + base] - lse2);
+        const float* m = a.ws + p.off_mass + base * p.CPT + c0;
+        if (VW == 4) {
+          const float4 v = *reinterpret_cast<const float4*>(m);
+          acc[0] = fmaf(v.x, f, acc[0]);
+          acc[1 % VW] = fmaf(v.y, f, acc[1 % VW]);
+          acc[2 % VW] = fmaf(v.z, f, acc[2 % VW]);
+          acc[3 % VW] = fmaf(v.w, f, acc[3 % VW]);
+        } else {
 #pragma unroll
-        for (int k = 0; k < VW; ++k) acc[k] = fmaf(m[k], f, acc[k]);
+          for (int k = 0; k < VW; ++k) acc[k] = fmaf(m[k], f, acc[k]);
+        }
       }
     }
   }
-  const float inv = 1.f / (float)p.Hq;
 #pragma unroll
-  for (int k = 0; k < VW; ++k) {
-    const int c = tile * p.CPT + c0 + k;
-    if (c < p.NC) a.chunk_score[(long long)t * p.NC + c] = acc[k] * inv;
+  for (int k = 0; k < VW; ++k) part[slice][t][k] = acc[k];
+  __syncthreads();
+  if (slice == 0 && t < p.T) {
+    const float inv = 1.f / (float)p.Hq;
+#pragma unroll
+    for (int k = 0; k < VW; ++k) {
+      float sum = 0.f;
+#pragma unroll
+      for (int q = 0; q < kScoreSlices; ++q) sum += part[q][t][k];
+      const int c = tile * p.CPT + c0 + k;
+      if (c < p.NC) a.chunk_score[(long long)t * p.NC + c] = sum * inv;
+    }
   }
+}
+
+template <int VW>
+cudaError_t launch_score(const AttnArgs& a, dim3 grid, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(64, kScoreSlices);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, score_kernel<VW>, a);
 }
 
 }  // namespace
@@ -181,14 +212,13 @@ cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches
   if (e != cudaSuccess) return e;
   if (p.want_score && p.NC > 0) {
     if (p.CPT >= 4) {
-      score_kernel<4><<<dim3(p.TPH, p.CPT / 4), 64, 0, st>>>(a);
+      e = launch_score<4>(a, dim3(p.TPH, p.CPT / 4), st);
     } else if (p.CPT == 2) {
-      score_kernel<2><<<dim3(p.TPH, 1), 64, 0, st>>>(a);
+      e = launch_score<2>(a, dim3(p.TPH, 1), st);
     } else {
-      score_kernel<1><<<dim3(p.TPH, 1), 64, 0, st>>>(a);
+      e = launch_score<1>(a, dim3(p.TPH, 1), st);
     }
     *n_launches += 1;
-    e = cudaGetLastError();
   }
   return e;
 }
