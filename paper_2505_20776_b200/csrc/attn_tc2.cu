@@ -185,7 +185,10 @@ __device__ __forceinline__ void commit_pair(uint64_t* bar) {
 #define SPX_EVT2(role, idx) do {} while (0)
 #endif
 
-template <bool SCORE>
+// SCORE: 0 no chunk sums; otherwise the class of the chunk size, so that each variant carries only the
+// code it runs (the loop of the exponentials is instruction-cache sensitive): 1 chunks of 32 keys,
+// 2 chunks of 64 or 128 keys, 3 chunks of fewer than 32 keys.
+template <int SCORE>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2Maps maps) {
   const AttnPlan& p = a.plan;
@@ -643,7 +646,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
 
           const float neg_m = -m_new;
           const uint64_t scale2x2 = pack_f32x2(scale2, scale2), neg_mx2 = pack_f32x2(neg_m, neg_m);
-          const bool score = SCORE && !is_tree;
+          const bool score = SCORE != 0 && !is_tree;
           float* mass = nullptr;
           if (score) {
             const long long rowbase = ((long long)prob * p.TPH + tile) * p.RB + rr;
@@ -678,9 +681,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             const float gs = (gs0 + gs1) + (gs2 + gs3);
             l += gs;
             if (score) {
-              if (p.C == 32) {
+              if (SCORE == 1) {
                 cg[c] = gs;
-              } else if (p.C > 32) {
+              } else if (SCORE == 2) {
                 csum += gs;
                 if ((((c + 1) * 32) & (p.C - 1)) == 0) {
                   mass[((c + 1) * 32) / p.C - 1] = csum;
@@ -705,7 +708,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           exp_chunk(s1, pk1, 1);
           exp_chunk(s2, pk2, 2);
           exp_chunk(s3, pk3, 3);
-          if (score && p.C == 32) *reinterpret_cast<float4*>(mass) = make_float4(cg[0], cg[1], cg[2], cg[3]);
+          if (SCORE == 1 && score) *reinterpret_cast<float4*>(mass) = make_float4(cg[0], cg[1], cg[2], cg[3]);
           // the P buffer is shared by all tiles: the PV of the previous tile must have read it
           ok = wait_prev_pv();
           if (!ok) break;
@@ -827,7 +830,7 @@ bool encode_q_map(CUtensorMap* m, const void* ptr, int T, int Hq, int G, long lo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool SCORE>
+template <int SCORE>
 cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
   static bool configured = false;
   if (!configured) {
@@ -870,7 +873,10 @@ cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launc
   }
   ok = ok && encode_q_map(&maps.q, a.Q, p.T, p.Hq, p.G, a.q_st, a.q_sh);
   if (!ok) return cudaErrorInvalidValue;
-  const cudaError_t e = p.want_score ? launch2<true>(a, maps, st) : launch2<false>(a, maps, st);
+  const cudaError_t e = !p.want_score ? launch2<0>(a, maps, st)
+                        : p.C == 32   ? launch2<1>(a, maps, st)
+                        : p.C > 32    ? launch2<2>(a, maps, st)
+                                      : launch2<3>(a, maps, st);
   *n_launches += 1;
   return e;
 }
