@@ -62,7 +62,7 @@ __device__ __forceinline__ void merge_batch(const float* __restrict__ pm, const 
 __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ AttnArgs a) {
   const AttnPlan& p = a.plan;
   sm100::pdl_launch_dependents();
-  sm100::pdl_wait();                               // the partial results of the attention kernel are complete
+  // everything that needs no global memory (indices, addresses, the output position) comes before the wait
   const int blocks_per_prob = p.RB / 32;
   const int prob = blockIdx.x / blocks_per_prob;
   const int rr0 = (blockIdx.x - prob * blocks_per_prob) * 32;
@@ -89,14 +89,17 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   const float* pl = a.ws + p.off_part_l + (long long)slot0 * p.RB + rr;
   const float* po = a.ws + p.off_part_o + (((long long)slot0 * nd4 + d4) * p.RB + rr) * 4;
   const long long ostride = (long long)nd4 * p.RB * 4;
+  const int t = r / p.G, h = g * p.G + r % p.G;
+  __nv_bfloat16* out = a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4;
+  float* lse_out = a.lse + (long long)h * p.T + t;
 
+  sm100::pdl_wait();                               // the partial results of the attention kernel are complete
   float M = -INFINITY, Z = 0.f;
   float4 acc0 = make_float4(0.f, 0.f, 0.f, 0.f), acc1 = acc0;
   for (int s = 0; s < nseg; s += 12) merge_batch<12>(pm, pl, po, ostride, p.RB, s, min(12, nseg - s), M, Z, acc0, acc1);
 
   const float inv = 1.f / Z;
-  const int t = r / p.G, h = g * p.G + r % p.G;
-  if (d4 == 0) a.lse[(long long)h * p.T + t] = (M + log2f(Z)) * kLn2;
+  if (d4 == 0) *lse_out = (M + log2f(Z)) * kLn2;
   __nv_bfloat162 b0 = __floats2bfloat162_rn(acc0.x * inv, acc0.y * inv);
   __nv_bfloat162 b1 = __floats2bfloat162_rn(acc0.z * inv, acc0.w * inv);
   __nv_bfloat162 b2 = __floats2bfloat162_rn(acc1.x * inv, acc1.y * inv);
@@ -106,7 +109,7 @@ __global__ void __launch_bounds__(256) merge_kernel(const __grid_constant__ Attn
   pk.y = *reinterpret_cast<uint32_t*>(&b1);
   pk.z = *reinterpret_cast<uint32_t*>(&b2);
   pk.w = *reinterpret_cast<uint32_t*>(&b3);
-  *reinterpret_cast<uint4*>(a.O + (long long)t * a.o_st + (long long)h * a.o_sh + d4 * 4) = pk;
+  *reinterpret_cast<uint4*>(out) = pk;
 }
 
 // Block = 64 tree nodes x kScoreSlices slices of the KV heads, for one key tile and one group of VW
