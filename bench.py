@@ -32,8 +32,8 @@ WORKLOAD_DESC = ("c2: Llama-3.1-8B layer shape (32 q heads / 8 kv heads / dim 12
                  "60-node level tree, 32 layers with independent K/V, scores from layer 31, chunk 32, top-k 32, "
                  "draft KV 8x128 gather of 1024 tokens")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_tc2_kernel), from the
-# ncu capture summarised in profiles/attn_tc2_kernel_c2_16k.md (67.92 MB read + 1.68 MB written).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 69597440
+# ncu capture summarised in profiles/attn_tc2_kernel_c2_16k.md (67.93 MB read + 2.03 MB written).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 69959424
 
 
 def load_peaks():
