@@ -17,6 +17,11 @@
  *     base pointers must be 16-byte aligned.
  *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
  *   - Calls that share a workspace or outputs must be ordered by the stream.
+ *   - The kernels of specext_verify_attn are launched with programmatic stream serialization, so
+ *     that the set-up of one overlaps the tail of the one before it in the stream; each of them
+ *     waits for that predecessor to complete (and its writes to be visible) before it reads or
+ *     writes global memory, so the stream order the caller sees is the usual one.  The calls can
+ *     be captured into CUDA graphs.
  */
 #ifndef SPECEXT_H_
 #define SPECEXT_H_
