@@ -13,8 +13,8 @@
 //
 // A softmax thread pulls its whole S row into registers and releases its S buffer at once, so the
 // S tiles run two key tiles ahead of the exponentials; P is kept in registers until the previous
-// PV has consumed the P buffer, and the PV of a tile is issued whenever its P is complete.  The two softmax warpgroups of a CTA take alternate
-// key tiles of the same 128 rows (one thread per row each); the running reference maximum of a
+// PV has consumed the P buffer, and the PV of a tile is issued whenever its P is complete.  The two
+// softmax warpgroups of a CTA take alternate key tiles of the same 128 rows (one thread per row each); the running reference maximum of a
 // row is handed from tile to tile through shared memory, each warpgroup keeps its own partial row
 // sum, and O is rescaled lazily by whichever warpgroup raises the maximum by more than 2^8.
 //
@@ -24,6 +24,10 @@
 // Barriers with arrivals from both CTAs live in the leader CTA; MMA completion is multicast to
 // both CTAs.  Every wait is bounded; an expired wait raises SPECEXT_ERR_TIMEOUT, and both CTAs
 // always reach the final cluster barrier before tensor memory is freed.
+//
+// The kernel is launched with programmatic stream serialization: barrier set-up, tensor-memory
+// allocation and the start-up cluster barrier run while the kernel before it in the stream finishes;
+// global memory is touched only after griddepcontrol.wait.
 #include "common.cuh"
 #include "sm100.cuh"
 
