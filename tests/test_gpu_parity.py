@@ -458,3 +458,16 @@ def test_back_to_back_calls_in_a_graph_share_a_workspace(cuda_device):
         O_ref, lse_ref, _ = oracle_layer(t_cpu, parent, w.prefix_len, w.chunk_size, None)
         assert np.abs(f64(O) - O_ref).max() <= O_ATOL
         assert np.abs(f64(lse) - lse_ref).max() <= LSE_ATOL
+    # the overlapped replays give, bit for bit, what one call at a time gives
+    graph_O = [O.clone() for O in outs]
+    graph_lse = [x.clone() for x in lses]
+    for _ in range(20):
+        g.replay()
+    torch.cuda.synchronize()
+    for t, O, lse, gO, gl in zip(layers, outs, lses, graph_O, graph_lse):
+        assert torch.equal(O, gO) and torch.equal(lse, gl)
+        O.zero_()
+        api.specext_verify_attn(d, t["Q"], t["K_prefix"], t["V_prefix"], t["K_tree"], t["V_tree"], par, O, lse,
+                                None, ws, status)
+        torch.cuda.synchronize()
+        assert torch.equal(O, gO) and torch.equal(lse, gl)
