@@ -136,6 +136,27 @@ def oracle_sample(w, parent, repeats):
     return t_attn, t_retr
 
 
+def replica_seed(base_seed: int, rank: int) -> int:
+    """Every replica (rank) verifies its own sequence."""
+    return base_seed + 1000 * rank
+
+
+def max_over_ranks(ms_total: float, world: int, device) -> float:
+    """The slowest rank's device time (all ranks get it); one process = its own time."""
+    if world <= 1:
+        return ms_total
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def us_per_layer(ms_total: float, steps: int, n_layers: int, world: int) -> float:
+    """Whole-job figure: every rank runs `steps` steps of `n_layers` layers in `ms_total`."""
+    return ms_total / steps * 1e3 / (n_layers * world)
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -210,7 +231,7 @@ def main():
     NL, L = w.n_layers, w.prefix_len
     parent_np = synth.make_tree(w)
     parent = torch.from_numpy(parent_np).to(dev)
-    seed = w.seed + 1000 * rank                      # every replica has its own sequence
+    seed = replica_seed(w.seed, rank)
     layers = [synth.make_layer(w, layer=i, device=dev, seed=seed) for i in range(NL)]
     dK, dV = synth.make_draft_kv(w, device=dev, seed=seed)
     hp = HotPath(w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_tree, w.chunk_size, w.top_k, L, device=dev)
@@ -367,12 +388,9 @@ def main():
         clocks = sampler.stop()
         assert hp.read_status() == 0, "device status set during the timed region"
 
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_per_step = ms_total / args.steps
-    value = ms_per_step * 1e3 / (NL * world)          # us per layer over all replicas
+    value = us_per_layer(ms_total, args.steps, NL, world)
 
     if rank == 0:
         peaks = load_peaks()
