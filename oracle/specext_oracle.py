@@ -172,14 +172,15 @@ def chunk_lengths(prefix_len: int, chunk_size: int) -> np.ndarray:
 
 
 def select_chunks(chunk_score_row: np.ndarray, prefix_len: int, chunk_size: int, k: int,
-                  key_dtype=np.float32) -> np.ndarray:
+                  key_dtype=np.float64) -> np.ndarray:
     """SelectChunks of Algorithm 1: indices of the top-k chunks, ascending.
 
     chunk_score_row [NC] holds summed probability per chunk; the ranking key is the chunk's
     average score, mass / len_c (Section 3.2.1).  Order: key descending, chunk index ascending
     among equal keys; the first min(k, NC) are kept and returned sorted by index.  The key is
-    formed in `key_dtype` (fp32 by default, the precision the library ranks in; the score row is
-    stored as fp32) so that the integer decision is taken in the same arithmetic on both sides.
+    formed in `key_dtype`: fp64 by default (the plain definition).  A test that hands the same
+    fp32 score row to the oracle and to another implementation may ask for np.float32, so that
+    the integer decision is taken in the same arithmetic on both sides.
     """
     score = np.asarray(chunk_score_row)
     NC = score.shape[0]

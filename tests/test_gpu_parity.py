@@ -99,7 +99,7 @@ def check_select_bit_exact(hp, score_row_f32, L, C, k):
     hp.select_chunks(0, L)
     assert hp.read_status() == 0
     nsel = int(hp.n_selected.item())
-    want = orc.select_chunks(score_row_f32, L, C, k)
+    want = orc.select_chunks(score_row_f32, L, C, k, key_dtype=np.float32)
     assert nsel == len(want) == min(k, NC)
     np.testing.assert_array_equal(hp.idx[:nsel].cpu().numpy(), want)
 
