@@ -116,7 +116,7 @@ def oracle_sample(w, parent, repeats):
     """Times the CPU oracle on one 16K layer (attention with scores) plus select + gather."""
     import numpy as np
     import torch
-    from paper_2505_20776_b200 import synth
+    from workloads import synth
     from oracle import specext_oracle as orc
     t = synth.make_layer(w, layer=w.n_layers - 1)
     dK, dV = synth.make_draft_kv(w)
@@ -170,7 +170,7 @@ def run_reference(args, rank):
     """The reference arm: the oracle as it stands, on the host cores, bounded sample per step."""
     if rank != 0:
         return
-    from paper_2505_20776_b200 import synth
+    from workloads import synth
     w = synth.WORKLOADS[WORKLOAD]
     parent = synth.make_tree(w)
     oracle_sample(w, parent, max(0, min(args.warmup, 1)))
@@ -212,7 +212,8 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2505_20776_b200 import api, build, synth
+    from paper_2505_20776_b200 import api, build
+    from workloads import synth
     from paper_2505_20776_b200.hotpath import HotPath
 
     if not torch.cuda.is_available():

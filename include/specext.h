@@ -17,7 +17,9 @@
  *     base pointers must be 16-byte aligned.
  *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
  *   - Calls that share a workspace or outputs must be ordered by the stream.
- *   - The kernels of specext_verify_attn are launched with programmatic stream serialization, so
+ *   - No call keeps state between calls or changes process-wide settings; a process may use the
+ *     library on several devices (the device current at the call is the one used).
+ *   - The kernels of these calls are launched with programmatic stream serialization, so
  *     that the set-up of one overlaps the tail of the one before it in the stream; each of them
  *     waits for that predecessor to complete (and its writes to be visible) before it reads or
  *     writes global memory, so the stream order the caller sees is the usual one.  The calls can
@@ -142,6 +144,21 @@ int specext_gather_kv(const void* draft_K, const void* draft_V, int32_t n_layers
                       int32_t* n_tokens_out, int32_t* device_status, void* cuda_stream);
 
 /*
+ * SelectChunks followed by UpdateDraftCache (the two steps Algorithm 1 runs back to back when
+ * doRetrieval is set) as ONE call: the same results, in idx, n_selected, K_out, V_out and
+ * n_tokens_out, as specext_select_chunks(..., k, ...) followed by specext_gather_kv(...,
+ * max_selected = k, ...), argument for argument.  For n_chunks <= 8192 and k <= 1024 it is a single
+ * kernel launch (every thread block repeats the deterministic selection and copies its share of the
+ * kept chunks, so no block waits for another); larger sizes run the two kernels.
+ */
+int specext_select_gather(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, const void* draft_K,
+                          const void* draft_V, int32_t n_layers, int32_t n_kv_heads, int32_t head_dim,
+                          int64_t stride_layer, int64_t stride_l, int64_t stride_h, int32_t* idx,
+                          int32_t* n_selected, void* K_out, void* V_out, int32_t* n_tokens_out,
+                          int32_t* device_status, void* cuda_stream);
+
+/*
  * Copies *device_status to the host after synchronising the stream and returns it (a bit set of
  * 1 << specext_status), or -SPECEXT_ERR_CUDA if the copy failed.  For tests and debugging; not
  * part of the asynchronous path.
@@ -168,7 +185,10 @@ int64_t specext_launch_count(void);
  *     SPECEXT_STATIC_SCRATCH_BYTES are rejected with SPECEXT_ERR_WORKSPACE; nothing is launched.
  *   - The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
  *   - The first call on each device looks up the device address of the array (with that device
- *     current) and caches it; make that first call outside of any stream capture.
+ *     current) and caches it; that look-up may be what makes the driver load the array onto the
+ *     device.  Make that first call at start-up: outside of any stream capture, and while the
+ *     device still has SPECEXT_STATIC_SCRATCH_BYTES to spare (a caller whose allocator has already
+ *     failed cannot count on a first call succeeding).
  *   - All calls on a device share the one array.  Calls must therefore not overlap on the GPU:
  *     order them on one stream (or by events); two calls running concurrently race on the scratch
  *     and both produce garbage.  Nothing in the array has to survive from one call to the next and
@@ -182,20 +202,6 @@ int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void
                                        const int32_t* parent, void* O, float* lse,
                                        float* chunk_score, int32_t* device_status,
                                        void* cuda_stream);
-
-/*
- * Process-wide tuning and cross-check switches (the paper has no counterpart).
- *   attn_kernel       : 0 = default: the paired-CTA tensor-core (tcgen05 cta_group::2) kernel for
- *                       head_dim 128 with more than 128 stacked query rows per KV head, else the
- *                       one-CTA tensor-core kernel; 2 / 3 = force the one-CTA / paired kernel
- *                       (3 falls back to 2 for shapes the paired kernel is not built for);
- *                       1 = the CUDA-core kernel, an independent on-device cross-check.
- *   min_tiles_per_cta : lower bound on the 128-key tiles one CTA processes (> 0 to change; fewer,
- *                       longer splits mean fewer partial results to merge).  Changes the
- *                       workspace size, so set it before querying specext_verify_attn_workspace.
- * Not thread-safe with respect to concurrent calls of the library.
- */
-int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta);
 
 #ifdef __cplusplus
 }

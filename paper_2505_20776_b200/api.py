@@ -42,15 +42,8 @@ class AttnDesc(ctypes.Structure):
 _LIB: Optional[ctypes.CDLL] = None
 
 
-def lib() -> ctypes.CDLL:
-    """Loads libspecext.so (built in-tree by build.py); raises if it is not there."""
-    global _LIB
-    if _LIB is not None:
-        return _LIB
-    path = _build.LIB_PATH
-    if not os.path.exists(path):
-        raise RuntimeError(f"{path} is missing: run `python -m paper_2505_20776_b200.build` "
-                           "(there is no fallback path)")
+def bind(path: str) -> ctypes.CDLL:
+    """Loads a build of the library and declares the signatures of include/specext.h on it."""
     L = ctypes.CDLL(path)
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     L.specext_verify_attn_workspace.restype = sz
@@ -64,16 +57,29 @@ def lib() -> ctypes.CDLL:
     L.specext_gather_kv.restype = ctypes.c_int
     L.specext_gather_kv.argtypes = [vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp, i32, vp, vp, vp,
                                     vp, vp]
+    L.specext_select_gather.restype = ctypes.c_int
+    L.specext_select_gather.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, i32, i64, i64, i64,
+                                        vp, vp, vp, vp, vp, vp, vp]
     L.specext_read_status.restype = ctypes.c_int
     L.specext_read_status.argtypes = [vp, vp]
     L.specext_status_string.restype = ctypes.c_char_p
     L.specext_status_string.argtypes = [ctypes.c_int]
     L.specext_launch_count.restype = i64
     L.specext_launch_count.argtypes = []
-    L.specext_set_tuning.restype = ctypes.c_int
-    L.specext_set_tuning.argtypes = [i32, i32]
-    _LIB = L
     return L
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libspecext.so (built in-tree by build.py); raises if it is not there."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run `python -m paper_2505_20776_b200.build` "
+                           "(there is no fallback path)")
+    _LIB = bind(path)
+    return _LIB
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -196,6 +202,35 @@ def specext_gather_kv(draft_K: torch.Tensor, draft_V: torch.Tensor, prefix_len: 
     _check(rc, "specext_gather_kv")
 
 
+def specext_select_gather(chunk_score: torch.Tensor, row: int, prefix_len: int, chunk_size: int, k: int,
+                          draft_K: torch.Tensor, draft_V: torch.Tensor, idx: torch.Tensor,
+                          n_selected: torch.Tensor, K_out: torch.Tensor, V_out: torch.Tensor,
+                          n_tokens_out: torch.Tensor, device_status: torch.Tensor) -> None:
+    """Enqueues SelectChunks + UpdateDraftCache as one call (one kernel launch for the usual sizes)."""
+    if chunk_score.dtype != torch.float32 or chunk_score.dim() != 2 or not chunk_score.is_contiguous():
+        raise ValueError("chunk_score must be a contiguous fp32 [n_tree][n_chunks] tensor")
+    if idx.dtype != torch.int32 or n_selected.dtype != torch.int32:
+        raise ValueError("idx and n_selected must be int32")
+    for t in (draft_K, draft_V):
+        if t.dtype != torch.bfloat16 or t.dim() != 4 or t.stride(3) != 1:
+            raise ValueError("draft K/V must be bf16 [layers][tokens][heads][dim]")
+    if draft_K.stride() != draft_V.stride():
+        raise ValueError("draft K and V must share strides")
+    n_tree, n_chunks = chunk_score.shape
+    nl, _, H, D = draft_K.shape
+    need = nl * k * chunk_size * H * D
+    if idx.numel() < min(k, n_chunks):
+        raise ValueError("idx is too small")
+    if not (K_out.is_contiguous() and V_out.is_contiguous()) or K_out.numel() < need or V_out.numel() < need:
+        raise ValueError("K_out/V_out must be contiguous and hold [layers][k*C][H][D]")
+    rc = lib().specext_select_gather(_ptr(chunk_score), n_tree, n_chunks, int(row), int(prefix_len),
+                                     int(chunk_size), int(k), _ptr(draft_K), _ptr(draft_V), nl, H, D,
+                                     draft_K.stride(0), draft_K.stride(1), draft_K.stride(2), _ptr(idx),
+                                     _ptr(n_selected), _ptr(K_out), _ptr(V_out), _ptr(n_tokens_out),
+                                     _ptr(device_status), _stream())
+    _check(rc, "specext_select_gather")
+
+
 def specext_read_status(device_status: torch.Tensor) -> int:
     """Synchronises the current stream and returns the device status bit set."""
     return int(lib().specext_read_status(_ptr(device_status), _stream()))
@@ -203,10 +238,6 @@ def specext_read_status(device_status: torch.Tensor) -> int:
 
 def specext_launch_count() -> int:
     return int(lib().specext_launch_count())
-
-
-def specext_set_tuning(attn_kernel: int = 0, min_tiles_per_cta: int = 0) -> None:
-    _check(lib().specext_set_tuning(int(attn_kernel), int(min_tiles_per_cta)), "specext_set_tuning")
 
 
 def status_bits(bits: int) -> Tuple[str, ...]:

@@ -11,6 +11,11 @@ cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int 
                               long long s_layer, long long s_l, long long s_h, const int32_t* idx,
                               const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
                               int32_t* n_tokens_out, int32_t* status, cudaStream_t st);
+bool spx_select_gather_fusable(int NC, int k);
+cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* dK, const void* dV, int n_layers,
+                                     int H, int D, int L, int C, long long s_layer, long long s_l, long long s_h,
+                                     int32_t* idx, int32_t* n_selected, void* K_out, void* V_out,
+                                     int32_t* n_tokens_out, int32_t* status, cudaStream_t st);
 
 // Scratch of the entry point that takes no workspace.  Part of the library image: resident on every
 // device that loads the library until the process exits.  Device code may name it directly; host
@@ -19,27 +24,37 @@ static __device__ __align__(256) unsigned char g_static_scratch[SPECEXT_STATIC_S
 
 namespace {
 
-constexpr int kMaxDevices = 64;
+constexpr int kMaxDevices = kSpxMaxDevices;
 std::atomic<void*> g_static_scratch_addr[kMaxDevices];
 
 std::atomic<long long> g_launches{0};
-std::atomic<int> g_attn_kernel{0};       // 0 = default, 1 = CUDA-core kernel, 2 = tensor-core kernel
-std::atomic<int> g_min_units{1};
-#ifdef SPX_TRACE
-long long* g_trace = nullptr;
-#endif         // lower bound on key tiles per CTA (tuning knob)
 
+// Kernel choice and split granularity.  The product library has one choice per shape; the test library
+// (SPECEXT_TESTING) can override it so that the tests reach the other kernels and coarser splits.
+#ifdef SPECEXT_TESTING
+std::atomic<int> g_attn_kernel{0};       // 0 = default, 1 = CUDA-core kernel, 2 = one-CTA kernel, 3 = paired kernel
+std::atomic<int> g_min_units{1};         // lower bound on key tiles per worker
+int tuning_kernel() { return g_attn_kernel.load(); }
+int tuning_min_units() { return g_min_units.load() < 1 ? 1 : g_min_units.load(); }
+#else
+constexpr int tuning_kernel() { return 0; }
+constexpr int tuning_min_units() { return 1; }
+#endif
+
+// Multiprocessor count of the current device (looked up once per device).
 int sm_count() {
-  static std::atomic<int> cached{0};
-  int v = cached.load();
-  if (v > 0) return v;
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+  static std::atomic<int> cached[kMaxDevices];
+  int dev = -1, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) {
     (void)cudaGetLastError();
     return 148;                           // B200; used only when no device is present (size queries)
   }
-  cached.store(n);
+  if (dev < kMaxDevices && (n = cached[dev].load()) > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  if (dev < kMaxDevices) cached[dev].store(n);
   return n;
 }
 
@@ -74,10 +89,10 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   const long long U = (long long)p.NP * p.UPP;
   if (U > (1ll << 30)) return SPECEXT_ERR_UNSUPPORTED;
   p.U = (int)U;
-  const int min_units = g_min_units.load() < 1 ? 1 : g_min_units.load();
-  const int want = g_attn_kernel.load();
+  const int min_units = tuning_min_units();
+  const int want = tuning_kernel();
   const bool pair_ok = p.D == 128 && p.RB == 256;       // what the paired-CTA kernel is built for
-  p.kernel = want == 1 ? 1 : ((want == 0 || want == 3) && pair_ok ? 3 : 2);
+  p.kernel = want == 1 ? 1 : ((want == 0 || want == 3) && pair_ok ? 3 : 2);   // want != 0 only in the test library
   if (p.kernel == 3) {
     // one worker = a cluster of two CTAs; every problem gets the same number of workers when possible
     const int n_workers = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
@@ -127,6 +142,23 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   return SPECEXT_OK;
 }
 
+int check_gather_args(const void* draft_K, const void* draft_V, int32_t n_layers, int32_t n_kv_heads,
+                      int32_t head_dim, int32_t prefix_len, int32_t chunk_size, int64_t stride_layer,
+                      int64_t stride_l, int64_t stride_h, int32_t max_selected, const void* K_out,
+                      const void* V_out, const int32_t* n_tokens_out) {
+  if (!draft_K || !draft_V || !K_out || !V_out || !n_tokens_out) return SPECEXT_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > 65535 || n_kv_heads < 1 || head_dim < 8 || (head_dim & 7) != 0 ||
+      prefix_len < 0 || chunk_size < 1 || max_selected < 1)
+    return SPECEXT_ERR_INVALID_ARG;
+  if (stride_h < head_dim || (stride_h & 7) || stride_l < head_dim || (stride_l & 7) || (stride_layer & 7) ||
+      stride_layer < 0)
+    return SPECEXT_ERR_INVALID_ARG;
+  if (!aligned16(draft_K) || !aligned16(draft_V) || !aligned16(K_out) || !aligned16(V_out))
+    return SPECEXT_ERR_INVALID_ARG;
+  if ((long long)max_selected * chunk_size > (1ll << 28)) return SPECEXT_ERR_UNSUPPORTED;
+  return SPECEXT_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -170,15 +202,14 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
   a.kv_sl = desc->kv_stride_l; a.kv_sh = desc->kv_stride_h;
   a.tkv_st = desc->tkv_stride_t; a.tkv_sh = desc->tkv_stride_h;
   a.o_st = desc->o_stride_t; a.o_sh = desc->o_stride_h;
-#ifdef SPX_TRACE
-  a.trace = g_trace;
-#endif
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int n = 0;
-  cudaError_t e = p.kernel == 1   ? spx_launch_attn_simt(a, st, &n)
-                  : p.kernel == 3 ? spx_launch_attn_tc2(a, st, &n)
-                                  : spx_launch_attn_tc(a, st, &n);
+  cudaError_t e;
+#ifdef SPECEXT_TESTING
+  if (p.kernel == 1) e = spx_launch_attn_simt(a, st, &n); else
+#endif
+  e = p.kernel == 3 ? spx_launch_attn_tc2(a, st, &n) : spx_launch_attn_tc(a, st, &n);
   if (e == cudaSuccess) e = spx_launch_merge(a, st, &n);
   g_launches.fetch_add(n);
   if (e != cudaSuccess) {
@@ -250,21 +281,49 @@ int specext_gather_kv(const void* draft_K, const void* draft_V, int32_t n_layers
                       int64_t stride_layer, int64_t stride_l, int64_t stride_h, const int32_t* idx,
                       const int32_t* n_selected, int32_t max_selected, void* K_out, void* V_out,
                       int32_t* n_tokens_out, int32_t* device_status, void* cuda_stream) {
-  if (!draft_K || !draft_V || !idx || !n_selected || !K_out || !V_out || !n_tokens_out)
-    return SPECEXT_ERR_INVALID_ARG;
-  if (n_layers < 1 || n_layers > 65535 || n_kv_heads < 1 || head_dim < 8 || (head_dim & 7) != 0 ||
-      prefix_len < 0 || chunk_size < 1 || max_selected < 1)
-    return SPECEXT_ERR_INVALID_ARG;
-  if (stride_h < head_dim || (stride_h & 7) || stride_l < head_dim || (stride_l & 7) || (stride_layer & 7) ||
-      stride_layer < 0)
-    return SPECEXT_ERR_INVALID_ARG;
-  if (!aligned16(draft_K) || !aligned16(draft_V) || !aligned16(K_out) || !aligned16(V_out))
-    return SPECEXT_ERR_INVALID_ARG;
-  if ((long long)max_selected * chunk_size > (1ll << 28)) return SPECEXT_ERR_UNSUPPORTED;
+  if (!idx || !n_selected) return SPECEXT_ERR_INVALID_ARG;
+  const int rc = check_gather_args(draft_K, draft_V, n_layers, n_kv_heads, head_dim, prefix_len, chunk_size,
+                                   stride_layer, stride_l, stride_h, max_selected, K_out, V_out, n_tokens_out);
+  if (rc != SPECEXT_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = spx_launch_gather(draft_K, draft_V, n_layers, n_kv_heads, head_dim, prefix_len, chunk_size,
                                     stride_layer, stride_l, stride_h, idx, n_selected, max_selected, K_out,
                                     V_out, n_tokens_out, device_status, st);
+  g_launches.fetch_add(1);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SPECEXT_ERR_CUDA;
+  }
+  return SPECEXT_OK;
+}
+
+int specext_select_gather(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, const void* draft_K,
+                          const void* draft_V, int32_t n_layers, int32_t n_kv_heads, int32_t head_dim,
+                          int64_t stride_layer, int64_t stride_l, int64_t stride_h, int32_t* idx,
+                          int32_t* n_selected, void* K_out, void* V_out, int32_t* n_tokens_out,
+                          int32_t* device_status, void* cuda_stream) {
+  const long long nc = chunk_size >= 1 && prefix_len >= 0 ? ((long long)prefix_len + chunk_size - 1) / chunk_size : -1;
+  const bool fuse = nc == n_chunks && n_tree >= 1 && row >= 0 && row < n_tree && k >= 1 && chunk_score &&
+                    spx_select_gather_fusable(n_chunks, k);
+  if (!fuse) {
+    // sizes the single launch is not built for, and every invalid argument, take the two calls
+    const int rc = specext_select_chunks(chunk_score, n_tree, n_chunks, row, prefix_len, chunk_size, k, idx,
+                                         n_selected, device_status, cuda_stream);
+    if (rc != SPECEXT_OK) return rc;
+    return specext_gather_kv(draft_K, draft_V, n_layers, n_kv_heads, head_dim, prefix_len, chunk_size, stride_layer,
+                             stride_l, stride_h, idx, n_selected, k, K_out, V_out, n_tokens_out, device_status,
+                             cuda_stream);
+  }
+  if (!idx || !n_selected) return SPECEXT_ERR_INVALID_ARG;
+  const int rc = check_gather_args(draft_K, draft_V, n_layers, n_kv_heads, head_dim, prefix_len, chunk_size,
+                                   stride_layer, stride_l, stride_h, k, K_out, V_out, n_tokens_out);
+  if (rc != SPECEXT_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const cudaError_t e = spx_launch_select_gather(chunk_score + (long long)row * n_chunks, k, draft_K, draft_V,
+                                                 n_layers, n_kv_heads, head_dim, prefix_len, chunk_size,
+                                                 stride_layer, stride_l, stride_h, idx, n_selected, K_out, V_out,
+                                                 n_tokens_out, device_status, st);
   g_launches.fetch_add(1);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
@@ -300,15 +359,16 @@ const char* specext_status_string(int status) {
 
 int64_t specext_launch_count(void) { return g_launches.load(); }
 
-#ifdef SPX_TRACE
-void specext_debug_set_trace(void* p) { g_trace = static_cast<long long*>(p); }
-#endif
 
-int specext_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta) {
+#ifdef SPECEXT_TESTING
+// Test library only: forces an attention kernel / a lower bound on key tiles per worker for every
+// later call in the process (see testing.h).
+int specext_test_set_tuning(int32_t attn_kernel, int32_t min_tiles_per_cta) {
   if (attn_kernel < 0 || attn_kernel > 3 || min_tiles_per_cta < 0) return SPECEXT_ERR_INVALID_ARG;
   g_attn_kernel.store(attn_kernel);
   if (min_tiles_per_cta > 0) g_min_units.store(min_tiles_per_cta);
   return SPECEXT_OK;
 }
+#endif
 
 }  // extern "C"

@@ -1,6 +1,6 @@
 // Plain CUDA-core (no tensor core) split-over-KV tree attention producing the same partial
-// results as the tensor-core kernel.  It covers head dimensions and group sizes the tcgen05
-// kernel is not built for, and serves as an independent on-device cross-check of that kernel.
+// results as the tensor-core kernels.  It is compiled into the test library only, where it serves as
+// an independent on-device cross-check of those kernels; the product library does not contain it.
 //
 // One CTA of 256 threads handles 64 query rows of one row block: thread = (row, quarter of D).
 // Per key tile of 128 tokens: pass 1 forms the scaled scores (log2 domain) of the tile in shared

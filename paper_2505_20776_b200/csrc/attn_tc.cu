@@ -78,9 +78,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
   Ctrl* ctl = reinterpret_cast<Ctrl*>(base + C::kBarOffset);
   volatile int* abort_flag = &ctl->abort_flag;
 
-#ifdef SPX_TRACE
-  const long long spx_t_start = clock64();
-#endif
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_mt = p.RB / 128;
   const int cta = blockIdx.x;
@@ -115,7 +112,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
     // ================================ TMA producer ==========================================
     setmaxnreg_dec<kRegsOther>();
     if (lane == 0) {
-      SPX_EVT(0, 0);
       uint32_t kvp = 0;
       int seg = 0;
       bool q_armed = false;
@@ -143,7 +139,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             for (int ds = 0; ds < DS; ++ds)
               tma_load_3d(ring + stage * C::kStageBytes + ds * kSubTileBytes, m, &ctl->kv_full[stage], ds * 64, g,
                           is_tree ? 0 : tile * SPX_TILE_KEYS);
-            SPX_EVT(0, 1 + kvp);
             ++kvp;
           }
         }
@@ -233,10 +228,8 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             ok = mbar_wait(&ctl->kv_full[ks], (kvc / NS) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            SPX_EVT(1, 0);
             for (int mt = 0; mt < n_mt; ++mt) issue_s(mt, ks);
             mma_commit(&ctl->kv_empty[ks]);
-            SPX_EVT(1, 1);
             ++kvc;
           }
           for (int i = 0; i < n && ok; ++i) {
@@ -248,13 +241,10 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             const uint32_t kph = (kvc / NS) & 1;
             ok = mbar_wait(&ctl->kv_full[vs], vph, abort_flag);
             for (int mt = 0; mt < n_mt && ok; ++mt) {
-              SPX_EVT(2, it * 4 + mt * 2);
               ok = mbar_wait(&ctl->p_full[mt], it & 1, abort_flag);
-              SPX_EVT(2, it * 4 + mt * 2 + 1);
               if (ok && i == 0 && seg > 0) ok = mbar_wait(&ctl->o_free[mt], (seg - 1) & 1, abort_flag);
               if (!ok) break;
               tc_fence_after();
-              SPX_EVT(1, 2 + it * 4 + mt * 2);
               issue_pv(mt, vs, i > 0 ? 1u : 0u);
               if (last) mma_commit(&ctl->o_done[mt]);
               if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[vs]);
@@ -267,7 +257,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
                 issue_s(mt, ks);
                 if (mt == n_mt - 1) mma_commit(&ctl->kv_empty[ks]);
               }
-              SPX_EVT(1, 3 + it * 4 + mt * 2);
             }
             if (has_next) ++kvc;
             ++it;
@@ -313,7 +302,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             ok = mbar_wait(&ctl->s_full[mt], it & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            if (lane == 0) SPX_EVT(4 + warp, it * 4);
 
             // the whole S row of this thread: 128 fp32 scores in registers
             uint32_t s0[32], s1[32], s2[32], s3[32];
@@ -350,7 +338,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
               t3 = fmax3(t3, __uint_as_float(s3[j]), __uint_as_float(s3[j + 1]));
             }
             const float tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
-            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 1);
             const float m_tile = tmax * scale2;
             float alpha = 1.f;
             bool rescale = false;
@@ -425,11 +412,9 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             exp_chunk(s1, 1);
             exp_chunk(s2, 2);
             exp_chunk(s3, 3);
-            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 2);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&ctl->p_full[mt]);
-            if (lane == 0) SPX_EVT(4 + warp, it * 4 + 3);
           }
           if (!ok) break;
 
@@ -437,7 +422,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           ok = mbar_wait(&ctl->o_done[mt], seg & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          if (lane == 0) SPX_EVT(4 + warp, 60 + (seg & 1) * 2);
           {
             const int slot = cta + prob;
             float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
@@ -456,7 +440,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             a.ws[p.off_part_m + (long long)slot * p.RB + rr] = m_used;
             a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l;
           }
-          if (lane == 0) SPX_EVT(4 + warp, 61 + (seg & 1) * 2);
           tc_fence_before();
           mbar_arrive(&ctl->o_free[mt]);
           u += tile_hi - tile_lo;
@@ -469,7 +452,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
   if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
   tc_fence_before();
   __syncthreads();
-  if (tid == 0) SPX_EVT(0, 63);
   if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(ctl->tmem_base, 512);
@@ -509,13 +491,9 @@ bool encode_map(CUtensorMap* m, const void* ptr, int D, long long n1, long long 
 
 template <int D, bool SCORE>
 cudaError_t launch(const AttnArgs& a, const TcMaps& maps, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg<D>::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SpxOncePerDevice once;
+  const cudaError_t ec = spx_opt_in_smem(attn_tc_kernel<D, SCORE>, Cfg<D>::kSmemBytes, &once);
+  if (ec != cudaSuccess) return ec;
   attn_tc_kernel<D, SCORE><<<a.plan.n_cta, kThreads, Cfg<D>::kSmemBytes, st>>>(a, maps);
   return cudaGetLastError();
 }

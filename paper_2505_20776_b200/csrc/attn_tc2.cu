@@ -179,15 +179,6 @@ __device__ __forceinline__ void commit_pair(uint64_t* bar) {
       : "memory");
 }
 
-#ifdef SPX_TRACE
-#define SPX_EVT2(role, idx)                                                                  \
-  do {                                                                                       \
-    if (a.trace && blockIdx.x < 2 && (idx) < 64)                                             \
-      a.trace[((int)blockIdx.x * 12 + (role)) * 64 + (idx)] = clock64() - spx_t_start;       \
-  } while (0)
-#else
-#define SPX_EVT2(role, idx) do {} while (0)
-#endif
 
 // SCORE: 0 no chunk sums; otherwise the class of the chunk size, so that each variant carries only the
 // code it runs (the loop of the exponentials is instruction-cache sensitive): 1 chunks of 32 keys,
@@ -203,9 +194,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   Ctrl* ctl = reinterpret_cast<Ctrl*>(base + kCtrlOffset);
   volatile int* abort_flag = &ctl->abort_flag;
 
-#ifdef SPX_TRACE
-  const long long spx_t_start = clock64();
-#endif
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // The cluster barrier that makes both CTAs' mbarriers visible is split: the producer warp
@@ -324,7 +312,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         arrive_expect_tx_cluster(bar, kStageBytes);
         tma_load_3d_pair(dst, m, bar, 0, g, key0);
         tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
-        SPX_EVT2(0, 2 * (int)kp);
         ++kp;
         return true;
       };
@@ -338,7 +325,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
         arrive_expect_tx_cluster(bar, kStageBytes);
         tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
-        SPX_EVT2(0, 2 * (int)vp + 1);
         ++vp;
         return true;
       };
@@ -431,7 +417,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
                           idesc_s, kk > 0 ? 1u : 0u);
             commit_pair(&ctl->s_full[w]);
             commit_pair(&ctl->k_empty[stage]);
-            SPX_EVT2(1, j);
             ++kc;
             ++n_w[w];
           }
@@ -461,7 +446,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             if (ok) ok = wait_c(&ctl->p_full, vc & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            SPX_EVT2(11, 2 * j);
             const uint32_t vb = ring_lo + stage * (kStageBytes >> 4);
             const uint32_t pa = tmem + kColP;
             mma_ts_pair(tmem + kColO, pa, vb, hi, idesc_o, j > 0 ? 1u : 0u);
@@ -471,7 +455,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             commit_pair(&ctl->v_empty[stage]);
             commit_pair(&ctl->pv_done[w]);
             if (j == n - 1) commit_pair(&ctl->o_done);
-            SPX_EVT2(11, 2 * j + 1);
             ++vc;
           }
           u += n;
@@ -555,11 +538,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           const bool is_tree = tile == p.TPH;
           const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
           const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
-          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1));
           ok = wait_c(&ctl->s_full[wg], n_mine & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
-          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 1);
           uint32_t s0[32], s1[32], s2[32], s3[32];
           tmem_ld32(s_addr, s0);
           tmem_ld32(s_addr + 32, s1);
@@ -613,7 +594,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           }
           ctl->m_row[row_t] = m_new;
           warp_arrive(&ctl->m_pub[wg], lane);
-          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 2);
           if (m_loc != m_new) {
             l *= (m_loc == -INFINITY) ? 0.f : ex2_approx(m_loc - m_new);
             m_loc = m_new;
@@ -723,7 +703,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           tmem_wait_st();
           tc_fence_before();
           warp_arrive_cluster(p_full_l, lane);
-          if (lane == 0) SPX_EVT2(2 + warp, 4 * (j >> 1) + 3);
           ++n_mine;
         }
         if (!ok) break;
@@ -738,11 +717,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const float m_fin = ctl->m_row[row_t];
         if (m_loc != m_fin) l *= (m_loc == -INFINITY) ? 0.f : ex2_approx(m_loc - m_fin);
         if (wg == 1) ctl->l_x[row_t] = l;
-        if (lane == 0) SPX_EVT2(2 + warp, 60);
         ok = wait_c(&ctl->o_done, seg & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        if (lane == 0) SPX_EVT2(2 + warp, 61);
         n_oth += wg == 0 ? (n >> 1) : ((n + 1) >> 1);
         warp_arrive(&ctl->epi[0], lane);                 // l_x visible; both warpgroups past their last tile
         ok = mbar_wait(&ctl->epi[0], seg & 1, abort_flag);
@@ -767,7 +744,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l + ctl->l_x[row_t];
           }
         }
-        if (lane == 0) SPX_EVT2(2 + warp, 62);
         u += n;
         if (u < unit_hi) {
           warp_arrive(&ctl->epi[1], lane);               // l_x and m_row may be reused
@@ -780,11 +756,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
 
   if (!ok && lane == 0) spx_raise(a.status, SPECEXT_ERR_TIMEOUT);
   tc_fence_before();
-  if (tid == 0) SPX_EVT2(10, 0);
   // The peer may still signal this CTA's barriers or read its halves, and tensor memory is freed by one
   // warp for all: everybody meets once more.  The partial results written above need no ordering here.
   cluster_sync_relaxed();
-  if (tid == 0) SPX_EVT2(10, 1);
   if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(ctl->tmem_base), "r"(512u) : "memory");
@@ -836,12 +810,9 @@ bool encode_q_map(CUtensorMap* m, const void* ptr, int T, int Hq, int G, long lo
 
 template <int SCORE>
 cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc2_kernel<SCORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SpxOncePerDevice once;
+  const cudaError_t ec = spx_opt_in_smem(attn_tc2_kernel<SCORE>, kSmemBytes, &once);
+  if (ec != cudaSuccess) return ec;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * a.plan.n_cta);
   cfg.blockDim = dim3(kThreads);

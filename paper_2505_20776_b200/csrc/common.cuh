@@ -23,20 +23,8 @@ struct AttnArgs {
   float* ws;
   int32_t* status;
   long long q_st, q_sh, kv_sl, kv_sh, tkv_st, tkv_sh, o_st, o_sh;
-#ifdef SPX_TRACE
-  long long* trace;   // timing trace of two CTAs (development builds only)
-#endif
 };
 
-#ifdef SPX_TRACE
-#define SPX_EVT(role, idx)                                                                              \
-  do {                                                                                                  \
-    if (a.trace && (blockIdx.x == 0 || blockIdx.x == 77) && (idx) < 64)                                 \
-      a.trace[((blockIdx.x ? 1 : 0) * 12 + (role)) * 64 + (idx)] = clock64() - spx_t_start;              \
-  } while (0)
-#else
-#define SPX_EVT(role, idx) do {} while (0)
-#endif
 
 __device__ __forceinline__ void spx_raise(int32_t* status, int code) {
   if (status) atomicOr(status, 1 << code);
@@ -66,8 +54,28 @@ __device__ __forceinline__ void spx_build_ancestors(const int32_t* __restrict__ 
   }
 }
 
+// A function attribute (the opt-in to large dynamic shared memory) belongs to the device's context, so
+// it is set once per (kernel, device), with the device current: `done` is the kernel's own table.
+constexpr int kSpxMaxDevices = 64;
+struct SpxOncePerDevice {
+  unsigned char done[kSpxMaxDevices] = {};
+};
+template <typename Kernel>
+cudaError_t spx_opt_in_smem(Kernel* kernel, int bytes, SpxOncePerDevice* once) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool cached = dev >= 0 && dev < kSpxMaxDevices;
+  if (cached && __atomic_load_n(&once->done[dev], __ATOMIC_ACQUIRE)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && cached) __atomic_store_n(&once->done[dev], (unsigned char)1, __ATOMIC_RELEASE);
+  return e;
+}
+
 // Launchers implemented in the kernel translation units; each returns the cudaError_t of its launch.
-cudaError_t spx_launch_attn_simt(const AttnArgs& a, cudaStream_t st, int* n_launches);
+#ifdef SPECEXT_TESTING
+cudaError_t spx_launch_attn_simt(const AttnArgs& a, cudaStream_t st, int* n_launches);   // cross-check kernel, test library only
+#endif
 cudaError_t spx_launch_attn_tc(const AttnArgs& a, cudaStream_t st, int* n_launches);
 cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launches);
 cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches);

@@ -195,12 +195,9 @@ cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches
   // kernel leaves first would take eight blocks each and a fraction of the SMs would do all the work:
   // an (unused) dynamic shared-memory request caps residency at one block per SM (measured: 1.1 us
   // per call faster than two per SM, which in turn was 2 us faster than no cap).
-  static bool configured = false;
-  if (!configured) {
-    const cudaError_t ec = cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemCap);
-    if (ec != cudaSuccess) return ec;
-    configured = true;
-  }
+  static SpxOncePerDevice once;
+  const cudaError_t ec = spx_opt_in_smem(merge_kernel, kMergeSmemCap, &once);
+  if (ec != cudaSuccess) return ec;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(256);

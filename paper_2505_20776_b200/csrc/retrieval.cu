@@ -9,10 +9,14 @@
 //
 // gather_kernel: 16-byte vector copy of the kept chunks of the draft K and V into the compact cache.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace {
 
 constexpr int kSelThreads = 1024;
+constexpr int kFusedThreads = 256;
+constexpr int kFusedMaxK = 1024;           // selected indices a fused block keeps in shared memory
+constexpr int kFusedMaxChunks = 8192;      // above this every block repeating the selection costs more than a launch
 
 __device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, int c, int NC, int L, int C) {
   const int len = (c == NC - 1) ? (L - c * C) : C;
@@ -21,26 +25,31 @@ __device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, i
   return __float_as_uint(x);
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ score, int NC, int L,
-                                                             int C, int k, int32_t* __restrict__ idx,
-                                                             int32_t* __restrict__ n_selected) {
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t s_prefix, s_need;
-  __shared__ uint32_t warp_tot[2][kSelThreads / 32];
-  __shared__ uint32_t carry[2];
+template <int NT>
+struct SelectSmem {
+  uint32_t hist[256];
+  uint32_t s_prefix, s_need;
+  uint32_t warp_tot[2][NT / 32];
+  uint32_t carry[2];
+};
+
+// Selection by one block of NT threads: writes the keff = min(k, NC) kept chunk indices, ascending,
+// to idx_out (global or shared memory).  Every thread of the block must call it.
+template <int NT>
+__device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __restrict__ score, int NC, int L,
+                                             int C, int keff, int32_t* idx_out) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int keff = min(k, NC);
 
   // ---- radix select of the keff-th largest key --------------------------------------------
   uint32_t prefix = 0, need = keff;        // `need` keys still to take among those matching prefix
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    if (tid < 256) hist[tid] = 0;
+    if (tid < 256) sm.hist[tid] = 0;
     __syncthreads();
-    for (int c = tid; c < NC; c += kSelThreads) {
+    for (int c = tid; c < NC; c += NT) {
       const uint32_t key = chunk_key(score, c, NC, L, C);
-      if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      if ((key & himask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
     if (warp == 0) {
@@ -48,7 +57,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
       uint32_t local[8], tot = 0;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        local[i] = hist[255 - (lane * 8 + i)];
+        local[i] = sm.hist[255 - (lane * 8 + i)];
         tot += local[i];
       }
       uint32_t incl = tot;
@@ -62,25 +71,25 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           if (before < need && need <= before + local[i]) {
-            s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + i)) << shift);
-            s_need = need - before;
+            sm.s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + i)) << shift);
+            sm.s_need = need - before;
           }
           before += local[i];
         }
       }
     }
     __syncthreads();
-    prefix = s_prefix;
-    need = s_need;
+    prefix = sm.s_prefix;
+    need = sm.s_need;
     __syncthreads();
   }
   const uint32_t theta = prefix;           // the keff-th largest key
   const uint32_t need_eq = need;           // how many keys equal to theta are kept (lowest indices)
 
   // ---- emit in ascending index order --------------------------------------------------------
-  if (tid == 0) carry[0] = carry[1] = 0;
+  if (tid == 0) sm.carry[0] = sm.carry[1] = 0;
   __syncthreads();
-  for (int base = 0; base < NC; base += kSelThreads) {
+  for (int base = 0; base < NC; base += NT) {
     const int c = base + tid;
     uint32_t key = 0;
     bool in = c < NC;
@@ -89,25 +98,35 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     const bool gt = in && key > theta;
     // exclusive count of `eq` before this chunk
     const uint32_t beq = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) warp_tot[0][warp] = __popc(beq);
+    if (lane == 0) sm.warp_tot[0][warp] = __popc(beq);
     __syncthreads();
-    uint32_t eq_before = carry[0] + __popc(beq & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) eq_before += warp_tot[0][w];
+    uint32_t eq_before = sm.carry[0] + __popc(beq & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) eq_before += sm.warp_tot[0][w];
     const bool keep = gt || (eq && eq_before < need_eq);
     const uint32_t bk = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) warp_tot[1][warp] = __popc(bk);
+    if (lane == 0) sm.warp_tot[1][warp] = __popc(bk);
     __syncthreads();
-    uint32_t pos = carry[1] + __popc(bk & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) pos += warp_tot[1][w];
-    if (keep && pos < (uint32_t)keff) idx[pos] = c;
+    uint32_t pos = sm.carry[1] + __popc(bk & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += sm.warp_tot[1][w];
+    if (keep && pos < (uint32_t)keff) idx_out[pos] = c;
     __syncthreads();
-    if (tid == kSelThreads - 1) {
-      carry[0] = eq_before + (eq ? 1u : 0u);
-      carry[1] = pos + (keep ? 1u : 0u);
+    if (tid == NT - 1) {
+      sm.carry[0] = eq_before + (eq ? 1u : 0u);
+      sm.carry[1] = pos + (keep ? 1u : 0u);
     }
     __syncthreads();
   }
-  if (tid == 0) *n_selected = keff;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ score, int NC, int L,
+                                                             int C, int k, int32_t* __restrict__ idx,
+                                                             int32_t* __restrict__ n_selected) {
+  __shared__ SelectSmem<kSelThreads> sm;
+  sm100::pdl_launch_dependents();
+  sm100::pdl_wait();                       // the scores are complete
+  const int keff = min(k, NC);
+  select_block<kSelThreads>(sm, score, NC, L, C, keff, idx);
+  if (threadIdx.x == 0) *n_selected = keff;
 }
 
 struct GatherArgs {
@@ -119,13 +138,39 @@ struct GatherArgs {
   int32_t* status;
   int n_layers, H, D, L, C, NC, max_selected, sub;
   long long s_layer, s_l, s_h;
+  // fused selection (select_gather_kernel only)
+  const float* score;
+  int32_t* idx_out;
+  int32_t* n_selected_out;
+  int k;
 };
+
+// Copies the tokens [o_lo, o_hi) of kept chunk number i (chunk index c) of one layer of K or V.
+__device__ __forceinline__ void gather_part(const GatherArgs& g, int i, int c, int part, int layer, int which) {
+  const int len = min(g.C, g.L - c * g.C);
+  const int tok_per_part = (g.C + g.sub - 1) / g.sub;
+  const int o_lo = part * tok_per_part, o_hi = min(len, o_lo + tok_per_part);
+  const int vpr = g.D / 8;                            // 16-byte vectors per head row
+  const int vpt = g.H * vpr;                          // per token
+  const __nv_bfloat16* src = g.src[which] + (long long)layer * g.s_layer;
+  __nv_bfloat16* dst = g.dst[which] + ((long long)layer * g.max_selected * g.C + (long long)i * g.C) * g.H * g.D;
+  const int nvec = max(0, o_hi - o_lo) * vpt;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    const int o = o_lo + v / vpt;
+    const int w = v - (v / vpt) * vpt;
+    const int hh = w / vpr, dv = w - hh * vpr;
+    const uint4 x = *reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o) * g.s_l + (long long)hh * g.s_h + dv * 8);
+    *reinterpret_cast<uint4*>(dst + ((long long)o * g.H + hh) * g.D + dv * 8) = x;
+  }
+}
 
 __global__ void __launch_bounds__(256) gather_kernel(const __grid_constant__ GatherArgs g) {
   const int i = blockIdx.x / g.sub;                  // which selected chunk
   const int part = blockIdx.x - i * g.sub;           // which slice of its tokens
   const int layer = blockIdx.y;
   const int which = blockIdx.z;                      // 0 = K, 1 = V
+  sm100::pdl_launch_dependents();
+  sm100::pdl_wait();                                 // idx and n_selected are complete
   int nsel = *g.n_selected;
   nsel = max(0, min(nsel, g.max_selected));
   if (blockIdx.x == 0 && layer == 0 && which == 0 && threadIdx.x == 0) {
@@ -142,42 +187,57 @@ __global__ void __launch_bounds__(256) gather_kernel(const __grid_constant__ Gat
     if (threadIdx.x == 0 && part == 0) spx_raise(g.status, SPECEXT_ERR_INVALID_ARG);
     return;
   }
-  const int len = min(g.C, g.L - c * g.C);
-  const int tok_per_part = (g.C + g.sub - 1) / g.sub;
-  const int o_lo = part * tok_per_part, o_hi = min(len, o_lo + tok_per_part);
-  const int vpr = g.D / 8;                            // 16-byte vectors per head row
-  const int vpt = g.H * vpr;                          // per token
-  const __nv_bfloat16* src = g.src[which] + (long long)layer * g.s_layer;
-  __nv_bfloat16* dst = g.dst[which] + ((long long)layer * g.max_selected * g.C + (long long)i * g.C) * g.H * g.D;
-  const int nvec = max(0, o_hi - o_lo) * vpt;
-  for (int v = threadIdx.x; v < nvec; v += 256) {
-    const int o = o_lo + v / vpt;
-    const int w = v - (v / vpt) * vpt;
-    const int hh = w / vpr, dv = w - hh * vpr;
-    const uint4 x = *reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o) * g.s_l + (long long)hh * g.s_h + dv * 8);
-    *reinterpret_cast<uint4*>(dst + ((long long)o * g.H + hh) * g.D + dv * 8) = x;
+  gather_part(g, i, c, part, layer, which);
+}
+
+// SelectChunks and UpdateDraftCache in one launch: every block repeats the (deterministic) selection
+// in its own shared memory and then copies its share of the kept chunks, so no block waits for
+// another; block (0, 0, 0) also writes idx, n_selected and n_tokens.
+__global__ void __launch_bounds__(kFusedThreads) select_gather_kernel(const __grid_constant__ GatherArgs g) {
+  __shared__ SelectSmem<kFusedThreads> sm;
+  __shared__ int32_t s_idx[kFusedMaxK];
+  const int i = blockIdx.x / g.sub;
+  const int part = blockIdx.x - i * g.sub;
+  const int layer = blockIdx.y;
+  const int which = blockIdx.z;
+  sm100::pdl_launch_dependents();
+  sm100::pdl_wait();                                 // the scores are complete
+  const int keff = min(g.k, g.NC);
+  if (i >= keff) return;                             // uniform for the block
+  select_block<kFusedThreads>(sm, g.score, g.NC, g.L, g.C, keff, s_idx);
+  __syncthreads();
+  if (blockIdx.x == 0 && layer == 0 && which == 0) {
+    for (int j = threadIdx.x; j < keff; j += kFusedThreads) g.idx_out[j] = s_idx[j];
+    if (threadIdx.x == 0) {
+      *g.n_selected_out = keff;
+      const int last = s_idx[keff - 1];
+      *g.n_tokens_out = (keff - 1) * g.C + min(g.C, g.L - last * g.C);
+    }
   }
+  gather_part(g, i, s_idx[i], part, layer, which);
 }
 
-}  // namespace
-
-cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
-                              int32_t* n_selected, cudaStream_t st) {
-  select_kernel<<<1, kSelThreads, 0, st>>>(score_row, NC, L, C, k, idx, n_selected);
-  return cudaGetLastError();
+cudaError_t launch_pdl(const void* kernel, dim3 grid, dim3 block, void** args, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
-cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
-                              long long s_layer, long long s_l, long long s_h, const int32_t* idx,
-                              const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
-                              int32_t* n_tokens_out, int32_t* status, cudaStream_t st) {
-  GatherArgs g;
+void fill_gather_args(GatherArgs& g, const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
+                      long long s_layer, long long s_l, long long s_h, int max_selected, void* K_out, void* V_out,
+                      int32_t* n_tokens_out, int32_t* status) {
   g.src[0] = static_cast<const __nv_bfloat16*>(dK);
   g.src[1] = static_cast<const __nv_bfloat16*>(dV);
   g.dst[0] = static_cast<__nv_bfloat16*>(K_out);
   g.dst[1] = static_cast<__nv_bfloat16*>(V_out);
-  g.idx = idx;
-  g.n_selected = n_selected;
   g.n_tokens_out = n_tokens_out;
   g.status = status;
   g.n_layers = n_layers; g.H = H; g.D = D; g.L = L; g.C = C;
@@ -189,7 +249,47 @@ cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int 
   sub = max(1, min(sub, C));
   g.sub = sub;
   g.s_layer = s_layer; g.s_l = s_l; g.s_h = s_h;
-  const dim3 grid(max_selected * sub, n_layers, 2);
-  gather_kernel<<<grid, 256, 0, st>>>(g);
-  return cudaGetLastError();
+  g.idx = nullptr; g.n_selected = nullptr;
+  g.score = nullptr; g.idx_out = nullptr; g.n_selected_out = nullptr; g.k = 0;
+}
+
+}  // namespace
+
+cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
+                              int32_t* n_selected, cudaStream_t st) {
+  void* args[] = {&score_row, &NC, &L, &C, &k, &idx, &n_selected};
+  return launch_pdl(reinterpret_cast<const void*>(select_kernel), dim3(1), dim3(kSelThreads), args, st);
+}
+
+cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
+                              long long s_layer, long long s_l, long long s_h, const int32_t* idx,
+                              const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
+                              int32_t* n_tokens_out, int32_t* status, cudaStream_t st) {
+  GatherArgs g;
+  fill_gather_args(g, dK, dV, n_layers, H, D, L, C, s_layer, s_l, s_h, max_selected, K_out, V_out, n_tokens_out,
+                   status);
+  g.idx = idx;
+  g.n_selected = n_selected;
+  void* args[] = {&g};
+  return launch_pdl(reinterpret_cast<const void*>(gather_kernel), dim3(max_selected * g.sub, n_layers, 2), dim3(256),
+                    args, st);
+}
+
+// True when SelectChunks + UpdateDraftCache of this size run as one launch.
+bool spx_select_gather_fusable(int NC, int k) { return NC >= 1 && NC <= kFusedMaxChunks && k <= kFusedMaxK; }
+
+cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* dK, const void* dV, int n_layers,
+                                     int H, int D, int L, int C, long long s_layer, long long s_l, long long s_h,
+                                     int32_t* idx, int32_t* n_selected, void* K_out, void* V_out,
+                                     int32_t* n_tokens_out, int32_t* status, cudaStream_t st) {
+  GatherArgs g;
+  fill_gather_args(g, dK, dV, n_layers, H, D, L, C, s_layer, s_l, s_h, k, K_out, V_out, n_tokens_out, status);
+  g.score = score_row;
+  g.idx_out = idx;
+  g.n_selected_out = n_selected;
+  g.k = k;
+  void* args[] = {&g};
+  const int keff = k < g.NC ? k : g.NC;
+  return launch_pdl(reinterpret_cast<const void*>(select_gather_kernel), dim3(keff * g.sub, n_layers, 2),
+                    dim3(kFusedThreads), args, st);
 }

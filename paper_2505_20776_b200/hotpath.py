@@ -22,25 +22,28 @@ class HotPath:
         self.C, self.k, self.max_prefix = chunk_size, top_k, max_prefix
         self.scale = softmax_scale
         self.device = torch.device(device)
-        dev = self.device
-        self.O = torch.empty(n_tree, n_q_heads, head_dim, dtype=torch.bfloat16, device=dev)
-        self.lse = torch.empty(n_q_heads, n_tree, dtype=torch.float32, device=dev)
+        self.O = self._alloc((n_tree, n_q_heads, head_dim), torch.bfloat16)
+        self.lse = self._alloc((n_q_heads, n_tree), torch.float32)
         self.max_chunks = -(-max_prefix // chunk_size)
-        self._score_flat = torch.empty(n_tree * max(1, self.max_chunks), dtype=torch.float32, device=dev)
-        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.idx = torch.full((max(1, top_k),), -1, dtype=torch.int32, device=dev)
-        self.n_selected = torch.zeros(1, dtype=torch.int32, device=dev)
-        self.n_tokens = torch.zeros(1, dtype=torch.int32, device=dev)
+        self._score_flat = self._alloc((n_tree * max(1, self.max_chunks),), torch.float32)
+        self.status = self._alloc((1,), torch.int32).zero_()
+        self.idx = self._alloc((max(1, top_k),), torch.int32).fill_(-1)
+        self.n_selected = self._alloc((1,), torch.int32).zero_()
+        self.n_tokens = self._alloc((1,), torch.int32).zero_()
         self.dl = draft_layers
         self.dH = draft_kv_heads or n_kv_heads
         self.dD = draft_head_dim or head_dim
         shape = (draft_layers, top_k * chunk_size, self.dH, self.dD)
-        self.K_compact = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
-        self.V_compact = torch.zeros(shape, dtype=torch.bfloat16, device=dev)
-        self._ws = torch.empty(0, dtype=torch.uint8, device=dev)
+        self.K_compact = self._alloc(shape, torch.bfloat16).zero_()
+        self.V_compact = self._alloc(shape, torch.bfloat16).zero_()
+        self._ws = self._alloc((0,), torch.uint8)
         self._desc_cache: Dict[tuple, api.AttnDesc] = {}
 
     # -- helpers -------------------------------------------------------------------------------
+    def _alloc(self, shape, dtype) -> torch.Tensor:
+        """Every device buffer of the sequence comes from here (a subclass may place them differently)."""
+        return torch.empty(shape, dtype=dtype, device=self.device)
+
     def n_chunks(self, prefix_len: int) -> int:
         return -(-prefix_len // self.C)
 
@@ -59,7 +62,7 @@ class HotPath:
             if need == 0:
                 raise api.SpecextError(2, "specext_verify_attn_workspace")
             if self._ws.numel() < need:
-                self._ws = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+                self._ws = self._alloc((need,), torch.uint8)
             self._desc_cache[key] = d
         return d
 
@@ -80,6 +83,12 @@ class HotPath:
     def gather_kv(self, draft_K: torch.Tensor, draft_V: torch.Tensor, prefix_len: int) -> None:
         api.specext_gather_kv(draft_K, draft_V, prefix_len, self.C, self.idx, self.n_selected, self.k,
                               self.K_compact, self.V_compact, self.n_tokens, self.status)
+
+    def select_gather(self, row: int, prefix_len: int, draft_K: torch.Tensor, draft_V: torch.Tensor) -> None:
+        """SelectChunks + UpdateDraftCache as one library call."""
+        api.specext_select_gather(self.chunk_score(prefix_len), row, prefix_len, self.C, self.k, draft_K, draft_V,
+                                  self.idx, self.n_selected, self.K_compact, self.V_compact, self.n_tokens,
+                                  self.status)
 
     def read_status(self) -> int:
         return api.specext_read_status(self.status)

@@ -29,6 +29,17 @@ def test_every_declared_symbol_is_exported(lib):
             "specext_verify_attn_workspace"} <= set(names)
     for n in names:
         assert hasattr(lib, n), f"{n} is declared in specext.h but not exported"
+    # test hooks and the cross-check kernel's switch live in the test library only
+    for n in ("specext_test_set_tuning", "specext_test_wait_timeout", "specext_set_tuning"):
+        assert not hasattr(lib, n)
+
+
+def test_test_library_builds_and_exports_its_hooks():
+    from tests.testing_lib import load_testing_lib
+    L = load_testing_lib()
+    assert hasattr(L, "specext_test_set_tuning") and hasattr(L, "specext_test_wait_timeout")
+    assert L.specext_test_set_tuning(7, 0) == 1
+    assert L.specext_test_wait_timeout(0, None, None) == 1
 
 
 def _desc(**kw):
@@ -68,5 +79,6 @@ def test_host_side_rejection_needs_no_gpu(lib):
     rc = lib.specext_verify_attn(ctypes.byref(d), *([None] * 9), None, 0, None, None)
     assert rc == 1                                            # null pointers
     assert lib.specext_select_chunks(None, 4, 8, 0, 256, 32, 4, None, None, None, None) == 1
+    assert lib.specext_select_gather(None, 4, 8, 0, 256, 32, 4, *([None] * 2), 1, 8, 128, 0, 1024, 128, *([None] * 7)) == 1
     assert lib.specext_status_string(4).decode().startswith("parent")
     assert lib.specext_launch_count() >= 0

@@ -2,7 +2,7 @@
 import numpy as np
 import torch
 
-from paper_2505_20776_b200 import synth
+from workloads import synth
 from oracle import specext_oracle as orc
 
 
