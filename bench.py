@@ -3,20 +3,24 @@
 
 One step = one verification pass of a 32-layer Llama-3.1-8B-shaped target over a 16K-token prefix
 and a 60-node draft tree (independent K/V per layer, 2.1 GB per step, so every layer comes from
-HBM), the last layer also producing chunk scores, followed by SelectChunks and UpdateDraftCache.
+HBM), the last layer also producing chunk scores, followed by SelectChunks + UpdateDraftCache.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-graph]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload all|c1|c2|c3|c4] [--no-graph]
 
-Prints ONE JSON line on rank 0.  With N > 1 (launched by torch.distributed.run) every rank runs an
-independent replica of the step on its own GPU; no collective is on the data path.
-`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+Prints ONE JSON line on rank 0.  The headline (`value`) is always workload c2; `--workload` chooses
+which of the other configurations are timed as well (key `workloads`: one verification-attention call
+and one scored call + retrieval per configuration, each replayed over enough distinct K/V buffers to
+stay out of L2).  With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica of the step on its own GPU; no collective is on the data path.  `--impl reference` times the
+CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
 import json
-import math
 import os
+import statistics
 import sys
 import threading
 import time
@@ -32,8 +36,9 @@ WORKLOAD_DESC = ("c2: Llama-3.1-8B layer shape (32 q heads / 8 kv heads / dim 12
                  "60-node level tree, 32 layers with independent K/V, scores from layer 31, chunk 32, top-k 32, "
                  "draft KV 8x128 gather of 1024 tokens")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_tc2_kernel), from the
-# ncu capture summarised in profiles/attn_tc2_kernel_c2_16k.md (67.93 MB read + 2.03 MB written).
+# ncu capture summarised in profiles/attn_tc2_kernel_c2_16k.md.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 69959424
+NOMINAL = {"hbm_gbs": 7700.0, "tf": 2250.0}            # B200 data-sheet figures, for context only
 
 
 def load_peaks():
@@ -52,14 +57,40 @@ def tree_depths(parent):
     return d
 
 
-def layer_work(w, parent, last_layer):
-    L, T, Hq, Hkv, D, C = w.prefix_len, w.n_tree, w.n_q_heads, w.n_kv_heads, w.head_dim, w.chunk_size
+def layer_work(w, parent, last_layer, prefix_len=None):
+    """Algorithmic bytes and flops of one verification-attention call (padding and split partials excluded)."""
+    L = w.prefix_len if prefix_len is None else prefix_len
+    T, Hq, Hkv, D, C = w.n_tree, w.n_q_heads, w.n_kv_heads, w.head_dim, w.chunk_size
     nbytes = 2 * L * Hkv * D * 2 + 2 * T * Hkv * D * 2 + 2 * T * Hq * D * 2 + Hq * T * 4
     if last_layer:
         nbytes += T * (-(-L // C)) * 4
     visible_tree = sum(d + 1 for d in tree_depths(parent))
     flops = 4 * Hq * D * (T * L + visible_tree)
     return nbytes, flops
+
+
+def retrieval_bytes(w, prefix_len=None):
+    """One score row read, the indices written, and the kept chunks of draft K and V read and written."""
+    L = w.prefix_len if prefix_len is None else prefix_len
+    nc = -(-L // w.chunk_size)
+    keff = min(w.top_k, nc)
+    h, d = w.draft_kv_heads or w.n_kv_heads, w.draft_head_dim or w.head_dim
+    return nc * 4 + keff * 4 + 4 * min(keff * w.chunk_size, L) * h * d * 2
+
+
+def tensor_peak(peaks, clocks):
+    """The bf16 peak that matches the run's own clock record: the burst figure when the sampled SM clock
+    stayed at its maximum, the sustained one (measured under the power cap at a lower clock) otherwise."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    if mhz and mx and mhz >= 0.97 * mx:
+        return peaks["tf_burst"], "burst (median SM clock at maximum during the timed region)"
+    return peaks["tf_sustained"], "sustained (SM clock below maximum, or no clock record)"
+
+
+def roof_times(nbytes, flops, peaks, tf):
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6
+    t_tc = flops / (tf * 1e12) * 1e6
+    return t_hbm, t_tc
 
 
 class ClockSampler:
@@ -109,12 +140,13 @@ class ClockSampler:
             self._thread.join()
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz,
+                "sm_mhz_min": s[0] if s else None,
+                "below_max_frac": (sum(1 for x in s if self.max_mhz and x < 0.97 * self.max_mhz) / len(s)) if s else None,
                 "reasons": sorted(self.reasons), "samples": len(s)}
 
 
 def oracle_sample(w, parent, repeats):
     """Times the CPU oracle on one 16K layer (attention with scores) plus select + gather."""
-    import numpy as np
     import torch
     from workloads import synth
     from oracle import specext_oracle as orc
@@ -167,7 +199,9 @@ def blas_threads():
 
 
 def run_reference(args, rank):
-    """The reference arm: the oracle as it stands, on the host cores, bounded sample per step."""
+    """The reference arm: the oracle as it stands, on the host cores.  One step of this arm is a bounded
+    sample of the workload's step: ONE of the 32 layers (with chunk scores) plus select + gather; that is
+    what `ms_per_step` times.  `value` spreads the retrieval over the 32 layers as the GPU arm does."""
     if rank != 0:
         return
     from workloads import synth
@@ -180,7 +214,8 @@ def run_reference(args, rank):
     sample = (f"per step: oracle verify_attn on 1 of the 32 layers (16K prefix, all 32 heads x 60 nodes, with "
               f"chunk scores) + select + gather; us/layer = t_attn + t_retrieval/32; {steps} steps timed")
     line = {"impl": "reference", "metric": METRIC, "value": per_layer_us, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": per_layer_us * w.n_layers / 1e3,
+            "steps": steps, "warmup": min(args.warmup, 1),
+            "ms_per_step": (sum(ta) + sum(tr)) / steps * 1e3, "sample_layers_per_step": 1,
             "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": WORKLOAD_DESC},
             "cpu_baseline": {"value": per_layer_us, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
@@ -189,12 +224,20 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+# Distinct K/V buffers a single-layer configuration rotates over so that no buffer is still in the
+# 126 MB L2 when its turn comes again (at least ~256 MB of other K/V in between).
+def copies_for(kv_bytes: int) -> int:
+    return max(4, -(-(384 << 20) // max(kv_bytes, 1)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="all", choices=["all", "c1", "c2", "c3", "c4"],
+                    help="which configurations are timed besides the c2 headline (c2 = headline only)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -241,23 +284,53 @@ def main():
     def step():
         for i in range(NL):
             hp.verify_attn(layers[i], parent, L, i == NL - 1)
-        hp.select_chunks(row, L)
-        hp.gather_kv(dK, dV, L)
+        hp.select_gather(row, L, dK, dV)
 
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def make_runner(fn):
+        """fn once eagerly (sizes the workspace), then captured in a graph unless --no-graph."""
+        fn()
+        stream.synchronize()
+        if args.no_graph:
+            return fn
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+        return g.replay
+
+    def timed(runner, reps, warm=2, per_replay=False):
+        """Device time in ms of `reps` back-to-back replays between two events (a barrier and a device
+        synchronisation on both sides).  With per_replay an event is recorded between consecutive replays
+        as well and the list of per-replay times is returned too; those events cost a little themselves."""
+        for _ in range(warm):
+            runner()
+        barrier()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1 if per_replay else 2)]
+        ev[0].record(stream)
+        for i in range(reps):
+            runner()
+            if per_replay:
+                ev[i + 1].record(stream)
+        if not per_replay:
+            ev[1].record(stream)
+        barrier()
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(reps)] if per_replay else None
+        return per, ev[0].elapsed_time(ev[-1])
+
     with torch.cuda.stream(stream):
         n0 = api.specext_launch_count()
         step()
         launches_per_step = api.specext_launch_count() - n0
         stream.synchronize()
-        graph = None
-        if not args.no_graph:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                step()
-        run = graph.replay if graph is not None else step
-
+        run = make_runner(step)
         for _ in range(args.warmup):
             run()
         stream.synchronize()
@@ -266,66 +339,21 @@ def main():
         sampler = ClockSampler(local_rank)
         sampler.start()
 
-        def barrier():
-            torch.cuda.synchronize()
-            if world > 1:
-                dist.barrier()
-                torch.cuda.synchronize()
-
         # ---- timed region: K steps, device timed ------------------------------------------
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(args.steps):
-            run()
-        e1.record(stream)
-        barrier()
-        ms_total = e0.elapsed_time(e1)
+        _, ms_total = timed(run, args.steps, warm=0)
+        # the same steps once more with an event after every replay, for the spread (median, minimum)
+        per_step_ms, _ = timed(run, args.steps, warm=0, per_replay=True)
 
-        # ---- roofline pass: only the score-less verification-attention calls (the dominant
-        # launch: attention kernel + merge), 31 distinct layers per replay so K/V comes from HBM
-        def attn_only():
+        # ---- the parts, each replayed alone the same way (reported, not part of `value`) ------
+        rsteps = max(3, min(args.steps, 50))
+
+        def part_us(fn, calls):
+            _, total = timed(make_runner(fn), rsteps)
+            return total / rsteps * 1e3 / calls
+
+        def attn_only():                                 # 31 distinct layers per replay: K/V comes from HBM
             for i in range(NL - 1):
                 hp.verify_attn(layers[i], parent, L, False)
-
-        attn_only()
-        stream.synchronize()
-        run_attn = attn_only
-        if not args.no_graph:
-            g2 = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g2, stream=stream):
-                attn_only()
-            run_attn = g2.replay
-        rsteps = max(3, min(args.steps, 50))
-        run_attn()
-        barrier()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(rsteps):
-            run_attn()
-        b.record(stream)
-        barrier()
-        attn_us_mean = a.elapsed_time(b) * 1e3 / (rsteps * (NL - 1))
-
-        # ---- the other parts, each timed alone the same way (reported, not part of `value`) --
-        def timed_us(fn, calls):
-            fn()
-            stream.synchronize()
-            runner = fn
-            if not args.no_graph:
-                gg = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(gg, stream=stream):
-                    fn()
-                runner = gg.replay
-            runner()
-            barrier()
-            x, y = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            x.record(stream)
-            for _ in range(rsteps):
-                runner()
-            y.record(stream)
-            barrier()
-            return x.elapsed_time(y) * 1e3 / (rsteps * calls)
 
         n_sc = min(NL, 8)                                # 8 distinct layers = 0.5 GB of K/V: from HBM
 
@@ -333,14 +361,65 @@ def main():
             for i in range(n_sc):
                 hp.verify_attn(layers[i], parent, L, True)
 
-        def retrieval():
-            hp.select_chunks(row, L)
-            hp.gather_kv(dK, dV, L)
+        n_rt = 16                                        # per graph, so that graph launches do not set the pace
 
-        parts = {"scoreless_layer_us": attn_us_mean, "score_layer_us": timed_us(score_layers, n_sc),
-                 "select_gather_us": timed_us(retrieval, 1),
-                 "note": "each part replayed alone; select+gather re-reads the same 8 MB (L2-resident)"}
+        def retrieval_one_call():
+            for _ in range(n_rt):
+                hp.select_gather(row, L, dK, dV)
+
+        def retrieval_two_calls():
+            for _ in range(n_rt):
+                hp.select_chunks(row, L)
+                hp.gather_kv(dK, dV, L)
+
+        attn_us = part_us(attn_only, NL - 1)
+        parts = {"scoreless_layer_us": attn_us, "score_layer_us": part_us(score_layers, n_sc),
+                 "select_gather_us": part_us(retrieval_one_call, n_rt),
+                 "select_then_gather_two_calls_us": part_us(retrieval_two_calls, n_rt),
+                 "note": "mean over back-to-back replays of each part alone; the retrieval parts re-read the same 8 MB "
+                         "(L2-resident)"}
         hp.verify_attn(layers[NL - 1], parent, L, True)  # leave the scores of the last layer in place
+
+        # ---- the other configurations ------------------------------------------------------
+        others = {}
+        which = [] if args.workload == "c2" or args.layers > 0 else (
+            ["c1", "c3", "c4"] if args.workload == "all" else [args.workload])
+        for name in which:
+            ww = synth.WORKLOADS[name]
+            par_np = synth.make_tree(ww)
+            par = torch.from_numpy(par_np).to(dev)
+            cap = ww.capacity or ww.prefix_len
+            lengths = synth.C3_LENGTHS if name == "c3" else (ww.prefix_len,)
+            per_tok = 2 * ww.n_kv_heads * ww.head_dim * 2
+            n_copies = copies_for(min(lengths) * per_tok)
+            # copy i is only ever read up to the longest length that still rotates over more than i copies
+            caps = [max(Lx for Lx in lengths if i < copies_for(Lx * per_tok)) for i in range(n_copies)]
+            bufs = [synth.make_layer(ww, layer=i, device=dev, capacity=min(cap, caps[i])) for i in range(n_copies)]
+            ddK, ddV = synth.make_draft_kv(ww, device=dev, capacity=cap)
+            hpo = HotPath(ww.n_q_heads, ww.n_kv_heads, ww.head_dim, ww.n_tree, ww.chunk_size, ww.top_k, cap,
+                          device=dev)
+            for Lx in lengths:
+                nb = min(n_copies, copies_for(Lx * per_tok))
+
+                def calls():
+                    for b in bufs[:nb]:
+                        hpo.verify_attn(b, par, Lx, False)
+
+                def scored_steps():                      # the in-place growth step: scored call + retrieval
+                    for b in bufs[:nb]:
+                        hpo.verify_attn(b, par, Lx, True)
+                        hpo.select_gather(row, Lx, ddK, ddV)
+
+                call_us = part_us(calls, nb)
+                step_us = part_us(scored_steps, nb)
+                nbytes, flops = layer_work(ww, par_np.tolist(), False, Lx)
+                others[name if name != "c3" else f"c3@{Lx}"] = {
+                    "prefix_len": Lx, "kv_copies_rotated": nb, "attn_call_us": call_us,
+                    "scored_call_plus_retrieval_us": step_us, "algorithmic_bytes": nbytes,
+                    "algorithmic_flops": flops}
+            assert hpo.read_status() == 0
+            del bufs, hpo, ddK, ddV
+            torch.cuda.empty_cache()
 
         # ---- end to end: host buffers, copies inside the timed region ----------------------
         e2e = None
@@ -364,26 +443,15 @@ def main():
                     hp.verify_attn(layers[i], parent, L, i == NL - 1)
                 dK.copy_(host_dK, non_blocking=True)
                 dV.copy_(host_dV, non_blocking=True)
-                hp.select_chunks(row, L)
-                hp.gather_kv(dK, dV, L)
+                hp.select_gather(row, L, dK, dV)
                 h_O.copy_(hp.O, non_blocking=True)
                 h_idx.copy_(hp.idx, non_blocking=True)
                 h_K.copy_(hp.K_compact, non_blocking=True)
                 h_V.copy_(hp.V_compact, non_blocking=True)
 
             e2e_step()
-            barrier()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for _ in range(args.e2e_steps):
-                e2e_step()
-            b.record(stream)
-            barrier()
-            e2e_ms = a.elapsed_time(b) / args.e2e_steps
-            if world > 1:
-                tt = torch.tensor([e2e_ms], device=dev)
-                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-                e2e_ms = float(tt.item())
+            _, e2e_total = timed(e2e_step, args.e2e_steps, warm=0)
+            e2e_ms = max_over_ranks(e2e_total / args.e2e_steps, world, dev)
             e2e = {"value": e2e_ms * 1e3 / (NL * world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                    "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
         clocks = sampler.stop()
@@ -395,36 +463,53 @@ def main():
 
     if rank == 0:
         peaks = load_peaks()
-        nbytes, flops = layer_work(w, parent_np.tolist(), False)
-        t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e6
-        t_tc = flops / (peaks["tf_sustained"] * 1e12) * 1e6
+        tf, tf_why = tensor_peak(peaks, clocks)
+        # whole step, per layer: the score-less layers, the scored layer and the retrieval
+        nb_plain, fl_plain = layer_work(w, parent_np.tolist(), False)
+        nb_last, fl_last = layer_work(w, parent_np.tolist(), True)
+        step_bytes = ((NL - 1) * nb_plain + nb_last + retrieval_bytes(w)) / NL
+        step_flops = ((NL - 1) * fl_plain + fl_last) / NL
+        t_hbm, t_tc = roof_times(step_bytes, step_flops, peaks, tf)
         t_roof = max(t_hbm, t_tc)
         if t_hbm >= t_tc:
-            roof = {"bound": "hbm", "achieved": nbytes / (attn_us_mean * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
+            roof = {"bound": "hbm", "achieved": step_bytes / (value * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s"}
         else:
-            roof = {"bound": "tensor", "achieved": flops / (attn_us_mean * 1e-6) / 1e12,
-                    "peak": peaks["tf_sustained"], "unit": "TFLOP/s"}
-        roof["frac"] = roof["achieved"] / roof["peak"]
+            roof = {"bound": "tensor", "achieved": step_flops / (value * 1e-6) / 1e12, "peak": tf, "unit": "TFLOP/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]          # = t_roof / value
         roof["traffic"] = NCU_TRAFFIC_BYTES_PER_LAUNCH
-        roof.update({"peak_source": peaks["source"] + (" (sustained bf16: kernel timed inside a long step)"
-                                                       if roof["bound"] == "tensor" else ""),
-                     "kernel": "verify-attention call of a score-less layer (attention + merge launches)",
-                     "launch_us_mean": attn_us_mean,
-                     "algorithmic_bytes": nbytes, "algorithmic_flops": flops,
-                     "achieved_gbs": nbytes / (attn_us_mean * 1e-6) / 1e9,
-                     "achieved_tflops": flops / (attn_us_mean * 1e-6) / 1e12,
-                     "t_hbm_us": t_hbm, "t_tensor_us": t_tc,
-                     "t_tensor_burst_us": flops / (peaks["tf_burst"] * 1e12) * 1e6,
-                     "t_roof_us": t_roof, "frac_of_roofline_time": t_roof / attn_us_mean})
+        ta_hbm, ta_tc = roof_times(nb_plain, fl_plain, peaks, tf)
+        roof.update({
+            "what": "whole step per layer: algorithmic bytes (or flops) of 31 score-less layers, the scored layer "
+                    "and select+gather, divided by 32 and by `value`; `traffic` is the attention kernel's DRAM "
+                    "bytes per launch from the ncu capture",
+            "peak_source": peaks["source"], "tensor_peak_used": tf_why,
+            "algorithmic_bytes_per_layer": step_bytes, "algorithmic_flops_per_layer": step_flops,
+            "t_hbm_us": t_hbm, "t_tensor_us": t_tc, "t_roof_us": t_roof,
+            "frac_tensor_burst": (step_flops / (peaks["tf_burst"] * 1e12) * 1e6) / value,
+            "frac_tensor_sustained": (step_flops / (peaks["tf_sustained"] * 1e12) * 1e6) / value,
+            "frac_hbm": t_hbm / value,
+            "frac_of_nominal": max(step_bytes / (NOMINAL["hbm_gbs"] * 1e9), step_flops / (NOMINAL["tf"] * 1e12))
+                               * 1e6 / value,
+            "attn_call": {"kernel": "verify-attention call of a score-less layer (attention + merge launches)",
+                          "launch_us_mean": attn_us, "algorithmic_bytes": nb_plain, "algorithmic_flops": fl_plain,
+                          "achieved_gbs": nb_plain / (attn_us * 1e-6) / 1e9,
+                          "achieved_tflops": fl_plain / (attn_us * 1e-6) / 1e12,
+                          "t_hbm_us": ta_hbm, "t_tensor_us": ta_tc, "frac": max(ta_hbm, ta_tc) / attn_us}})
+        for o in others.values():
+            th, tt = roof_times(o["algorithmic_bytes"], o["algorithmic_flops"], peaks, tf)
+            o.update({"t_hbm_us": th, "t_tensor_us": tt, "frac": max(th, tt) / o["attn_call_us"]})
+        per_layer = sorted(m * 1e3 / NL for m in per_step_ms)
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": WORKLOAD_DESC, "l2": "inputs larger than L2 (2.1 GB of K/V read per step)",
-                           "cuda_graph": graph is not None, "replicas": world,
+                           "cuda_graph": not args.no_graph, "replicas": world,
                            **({"profiling_layers": NL} if args.layers > 0 else {})},
+                "per_replay": {"median": statistics.median(per_layer), "min": per_layer[0], "unit": UNIT,
+                               "note": "separate pass of the same steps with an event after every replay"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-                "roofline": roof, "parts": parts}
+                "roofline": roof, "parts": parts, "workloads": others}
         if world == 1 and not args.no_cpu_baseline:
             ta, tr = oracle_sample(w, parent_np, 3)
             cpu_us = (sum(ta) / len(ta) + sum(tr) / len(tr) / NL) * 1e6

@@ -25,12 +25,15 @@ __device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, i
   return __float_as_uint(x);
 }
 
+constexpr int kKeyCache = 2048;            // ranking keys kept in shared memory (more chunks: recomputed per pass)
+
 template <int NT>
 struct SelectSmem {
   uint32_t hist[256];
   uint32_t s_prefix, s_need;
   uint32_t warp_tot[2][NT / 32];
   uint32_t carry[2];
+  uint32_t keys[kKeyCache];
 };
 
 // Selection by one block of NT threads: writes the keff = min(k, NC) kept chunk indices, ascending,
@@ -39,6 +42,11 @@ template <int NT>
 __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __restrict__ score, int NC, int L,
                                              int C, int keff, int32_t* idx_out) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // one load and one division per chunk when the keys fit in shared memory
+  const bool cached = NC <= kKeyCache;
+  if (cached)
+    for (int c = tid; c < NC; c += NT) sm.keys[c] = chunk_key(score, c, NC, L, C);
+  auto key_of = [&](int c) -> uint32_t { return cached ? sm.keys[c] : chunk_key(score, c, NC, L, C); };
 
   // ---- radix select of the keff-th largest key --------------------------------------------
   uint32_t prefix = 0, need = keff;        // `need` keys still to take among those matching prefix
@@ -48,7 +56,7 @@ __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __
     if (tid < 256) sm.hist[tid] = 0;
     __syncthreads();
     for (int c = tid; c < NC; c += NT) {
-      const uint32_t key = chunk_key(score, c, NC, L, C);
+      const uint32_t key = key_of(c);
       if ((key & himask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
@@ -93,7 +101,7 @@ __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __
     const int c = base + tid;
     uint32_t key = 0;
     bool in = c < NC;
-    if (in) key = chunk_key(score, c, NC, L, C);
+    if (in) key = key_of(c);
     const bool eq = in && key == theta;
     const bool gt = in && key > theta;
     // exclusive count of `eq` before this chunk
@@ -155,12 +163,24 @@ __device__ __forceinline__ void gather_part(const GatherArgs& g, int i, int c, i
   const __nv_bfloat16* src = g.src[which] + (long long)layer * g.s_layer;
   __nv_bfloat16* dst = g.dst[which] + ((long long)layer * g.max_selected * g.C + (long long)i * g.C) * g.H * g.D;
   const int nvec = max(0, o_hi - o_lo) * vpt;
-  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
-    const int o = o_lo + v / vpt;
-    const int w = v - (v / vpt) * vpt;
-    const int hh = w / vpr, dv = w - hh * vpr;
-    const uint4 x = *reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o) * g.s_l + (long long)hh * g.s_h + dv * 8);
-    *reinterpret_cast<uint4*>(dst + ((long long)o * g.H + hh) * g.D + dv * 8) = x;
+  // four vectors per thread and round: all loads are issued before the first store
+  for (int v0 = threadIdx.x; v0 < nvec; v0 += 4 * blockDim.x) {
+    uint4 x[4];
+    long long off[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int v = v0 + q * blockDim.x;
+      if (v < nvec) {
+        const int o = o_lo + v / vpt;
+        const int w = v - (v / vpt) * vpt;
+        const int hh = w / vpr, dv = w - hh * vpr;
+        x[q] = *reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o) * g.s_l + (long long)hh * g.s_h + dv * 8);
+        off[q] = ((long long)o * g.H + hh) * g.D + dv * 8;
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (v0 + q * blockDim.x < nvec) *reinterpret_cast<uint4*>(dst + off[q]) = x[q];
   }
 }
 
