@@ -372,10 +372,36 @@ def main():
                 hp.select_chunks(row, L)
                 hp.gather_kv(dK, dV, L)
 
+        # draft-side attention on the compact cache the retrieval just wrote (a 10-node draft step of an
+        # EAGLE-class layer: 32 query heads on the cache's 8 KV heads), its length read on the device
+        wdr = synth.Workload("draft", w.n_q_heads, dK.shape[2], dK.shape[3], w.top_k * w.chunk_size, 10, w.chunk_size,
+                             1, "uniform", "normal", seed=seed + 7)
+        tdr = synth.make_layer(wdr, device=dev)
+        pdr_np = synth.make_tree(wdr)
+        pdr = torch.from_numpy(pdr_np).to(dev)
+        O_dr = torch.empty_like(tdr["Q"])
+        lse_dr = torch.empty(wdr.n_q_heads, wdr.n_tree, dtype=torch.float32, device=dev)
+        d_dr = api.make_attn_desc(tdr["Q"], hp.K_compact[0], tdr["K_tree"], O_dr, wdr.prefix_len, w.chunk_size)
+        ws_dr = torch.empty(api.specext_verify_attn_workspace(d_dr), dtype=torch.uint8, device=dev)
+
+        def draft_attn():
+            for _ in range(n_rt):
+                api.specext_draft_attn(d_dr, tdr["Q"], hp.K_compact[0], hp.V_compact[0], hp.n_tokens, tdr["K_tree"],
+                                       tdr["V_tree"], pdr, O_dr, lse_dr, ws_dr, hp.status)
+
+        def retrieval_then_draft():
+            for _ in range(n_rt):
+                hp.select_gather(row, L, dK, dV)
+                api.specext_draft_attn(d_dr, tdr["Q"], hp.K_compact[0], hp.V_compact[0], hp.n_tokens, tdr["K_tree"],
+                                       tdr["V_tree"], pdr, O_dr, lse_dr, ws_dr, hp.status)
+
         attn_us = part_us(attn_only, NL - 1)
         parts = {"scoreless_layer_us": attn_us, "score_layer_us": part_us(score_layers, n_sc),
                  "select_gather_us": part_us(retrieval_one_call, n_rt),
                  "select_then_gather_two_calls_us": part_us(retrieval_two_calls, n_rt),
+                 "draft_attn_us": part_us(draft_attn, n_rt),
+                 "select_gather_then_draft_attn_us": part_us(retrieval_then_draft, n_rt),
+                 "draft_attn_algorithmic_bytes": layer_work(wdr, pdr_np.tolist(), False)[0],
                  "note": "mean over back-to-back replays of each part alone; the retrieval parts re-read the same 8 MB "
                          "(L2-resident)"}
         hp.verify_attn(layers[NL - 1], parent, L, True)  # leave the scores of the last layer in place
@@ -496,6 +522,7 @@ def main():
                           "achieved_gbs": nb_plain / (attn_us * 1e-6) / 1e9,
                           "achieved_tflops": fl_plain / (attn_us * 1e-6) / 1e12,
                           "t_hbm_us": ta_hbm, "t_tensor_us": ta_tc, "frac": max(ta_hbm, ta_tc) / attn_us}})
+        parts["draft_attn_t_hbm_us"] = parts["draft_attn_algorithmic_bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
         for o in others.values():
             th, tt = roof_times(o["algorithmic_bytes"], o["algorithmic_flops"], peaks, tf)
             o.update({"t_hbm_us": th, "t_tensor_us": tt, "frac": max(th, tt) / o["attn_call_us"]})

@@ -144,6 +144,32 @@ int specext_gather_kv(const void* draft_K, const void* draft_V, int32_t n_layers
                       int32_t* n_tokens_out, int32_t* device_status, void* cuda_stream);
 
 /*
+ * Attention of the DRAFT model over the compact cache that UpdateDraftCache wrote (Section 3.2.1,
+ * "Method Overview": the draft model generates its candidate tokens on the reduced cache of the
+ * selected chunks; Appendix D: about 1K to 2K tokens).  The arithmetic is that of
+ * specext_verify_attn -- tree nodes (or a single decode token, n_tree = 1) attend to the cached
+ * tokens and to their own ancestors, split over the KV length and merged by log-sum-exp -- but
+ * the number of cached tokens is read ON THE DEVICE, so that select -> gather -> draft attention
+ * replay as one CUDA graph with no host round trip in between.
+ *
+ *   desc->prefix_len : capacity of the compact cache in tokens (k * chunk_size), the upper bound of
+ *                      *n_tokens; desc->want_chunk_score must be 0; desc->chunk_size is not used
+ *                      (give any valid value).
+ *   K_cache, V_cache : bf16 [>= capacity][n_kv_heads][head_dim], strides desc->kv_stride_*, e.g. one
+ *                      layer of the K_out / V_out of specext_gather_kv.
+ *   n_tokens         : int32 [1] in DEVICE memory (the n_tokens_out of specext_gather_kv); values
+ *                      outside [0, capacity] are clamped.  Cache rows at and beyond *n_tokens are
+ *                      never used, whatever they hold (NaN included).
+ *   everything else  : as in specext_verify_attn; the workspace size is
+ *                      specext_verify_attn_workspace(desc).
+ * The work is laid out for the capacity; with a shorter cache some thread blocks find nothing to do.
+ */
+int specext_draft_attn(const specext_attn_desc* desc, const void* Q, const void* K_cache,
+                       const void* V_cache, const int32_t* n_tokens, const void* K_tree,
+                       const void* V_tree, const int32_t* parent, void* O, float* lse, void* workspace,
+                       size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
+
+/*
  * SelectChunks followed by UpdateDraftCache (the two steps Algorithm 1 runs back to back when
  * doRetrieval is set) as ONE call: the same results, in idx, n_selected, K_out, V_out and
  * n_tokens_out, as specext_select_chunks(..., k, ...) followed by specext_gather_kv(...,

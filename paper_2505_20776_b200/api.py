@@ -57,6 +57,8 @@ def bind(path: str) -> ctypes.CDLL:
     L.specext_gather_kv.restype = ctypes.c_int
     L.specext_gather_kv.argtypes = [vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp, i32, vp, vp, vp,
                                     vp, vp]
+    L.specext_draft_attn.restype = ctypes.c_int
+    L.specext_draft_attn.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9 + [vp, sz, vp, vp]
     L.specext_select_gather.restype = ctypes.c_int
     L.specext_select_gather.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, i32, i64, i64, i64,
                                         vp, vp, vp, vp, vp, vp, vp]
@@ -143,6 +145,22 @@ def specext_verify_attn(desc: AttnDesc, Q: torch.Tensor, K_prefix: torch.Tensor,
                                    _ptr(workspace), workspace.numel() * workspace.element_size(),
                                    _ptr(device_status), _stream())
     _check(rc, "specext_verify_attn")
+
+
+def specext_draft_attn(desc: AttnDesc, Q: torch.Tensor, K_cache: torch.Tensor, V_cache: torch.Tensor,
+                       n_tokens: torch.Tensor, K_tree: torch.Tensor, V_tree: torch.Tensor, parent: torch.Tensor,
+                       O: torch.Tensor, lse: torch.Tensor, workspace: torch.Tensor,
+                       device_status: torch.Tensor) -> None:
+    """Enqueues the draft model's attention over a compact cache whose length is an int32 on the device."""
+    if V_cache.stride() != K_cache.stride() or V_tree.stride() != K_tree.stride():
+        raise ValueError("V tensors must have the strides of the matching K tensors")
+    if (parent.dtype != torch.int32 or lse.dtype != torch.float32 or device_status.dtype != torch.int32 or
+            n_tokens.dtype != torch.int32):
+        raise ValueError("parent/device_status/n_tokens must be int32 and lse fp32")
+    rc = lib().specext_draft_attn(ctypes.byref(desc), _ptr(Q), _ptr(K_cache), _ptr(V_cache), _ptr(n_tokens),
+                                  _ptr(K_tree), _ptr(V_tree), _ptr(parent), _ptr(O), _ptr(lse), _ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _ptr(device_status), _stream())
+    _check(rc, "specext_draft_attn")
 
 
 STATIC_SCRATCH_BYTES = 32 << 20

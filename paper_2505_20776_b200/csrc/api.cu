@@ -169,15 +169,23 @@ size_t specext_verify_attn_workspace(const specext_attn_desc* desc) {
   return (size_t)p.total_floats * sizeof(float);
 }
 
-int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void* K_prefix,
-                        const void* V_prefix, const void* K_tree, const void* V_tree,
-                        const int32_t* parent, void* O, float* lse, float* chunk_score,
-                        void* workspace, size_t workspace_bytes, int32_t* device_status,
-                        void* cuda_stream) {
+}  // extern "C"
+
+namespace {
+
+// Checks, plan and launches shared by specext_verify_attn (prefix_len_dev == null) and
+// specext_draft_attn (the prefix length is read on the device, desc->prefix_len is its upper bound).
+int run_attn(const specext_attn_desc* desc, const void* Q, const void* K_prefix, const void* V_prefix,
+             const void* K_tree, const void* V_tree, const int32_t* parent, const int32_t* prefix_len_dev,
+             void* O, float* lse, float* chunk_score, void* workspace, size_t workspace_bytes,
+             int32_t* device_status, void* cuda_stream) {
   AttnArgs a;
   const int rc = build_plan(desc, &a.plan);
   if (rc != SPECEXT_OK) return rc;
   const AttnPlan& p = a.plan;
+  if (prefix_len_dev && (p.want_score || p.kernel == 1 || (reinterpret_cast<uintptr_t>(prefix_len_dev) & 3u) != 0))
+    return p.want_score ? SPECEXT_ERR_INVALID_ARG : (p.kernel == 1 ? SPECEXT_ERR_UNSUPPORTED : SPECEXT_ERR_INVALID_ARG);
+  a.L_dev = prefix_len_dev;
   if (!Q || !K_tree || !V_tree || !parent || !O || !lse || !workspace) return SPECEXT_ERR_INVALID_ARG;
   if (p.L > 0 && (!K_prefix || !V_prefix)) return SPECEXT_ERR_INVALID_ARG;
   if (p.want_score && p.NC > 0 && !chunk_score) return SPECEXT_ERR_INVALID_ARG;
@@ -217,6 +225,28 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
     return SPECEXT_ERR_CUDA;
   }
   return SPECEXT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void* K_prefix,
+                        const void* V_prefix, const void* K_tree, const void* V_tree,
+                        const int32_t* parent, void* O, float* lse, float* chunk_score,
+                        void* workspace, size_t workspace_bytes, int32_t* device_status,
+                        void* cuda_stream) {
+  return run_attn(desc, Q, K_prefix, V_prefix, K_tree, V_tree, parent, nullptr, O, lse, chunk_score, workspace,
+                  workspace_bytes, device_status, cuda_stream);
+}
+
+int specext_draft_attn(const specext_attn_desc* desc, const void* Q, const void* K_cache,
+                       const void* V_cache, const int32_t* n_tokens, const void* K_tree,
+                       const void* V_tree, const int32_t* parent, void* O, float* lse, void* workspace,
+                       size_t workspace_bytes, int32_t* device_status, void* cuda_stream) {
+  if (!n_tokens) return SPECEXT_ERR_INVALID_ARG;
+  return run_attn(desc, Q, K_cache, V_cache, K_tree, V_tree, parent, n_tokens, O, lse, nullptr, workspace,
+                  workspace_bytes, device_status, cuda_stream);
 }
 
 int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void* Q,

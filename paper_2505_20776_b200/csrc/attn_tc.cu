@@ -54,6 +54,7 @@ struct Cfg {
 
 struct Ctrl {
   uint64_t q_full, q_free, drain;
+  uint64_t v_rag;                 // a V tile whose tail rows must be cleared has landed (device-side length)
   uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
   uint64_t kv_full[8], kv_empty[8];
   unsigned long long anc[64];
@@ -62,7 +63,9 @@ struct Ctrl {
   int abort_flag;
 };
 
-template <int D, bool SCORE>
+// DEVLEN: the prefix length is read from device memory (a.L_dev) and may be shorter than the planned
+// capacity p.L; the instantiation without it carries none of that code.
+template <int D, bool SCORE, bool DEVLEN>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMaps maps) {
   using C = Cfg<D>;
@@ -87,6 +90,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
     mbar_init(&ctl->q_full, 1);
     mbar_init(&ctl->q_free, 1);
     mbar_init(&ctl->drain, 1);
+    mbar_init(&ctl->v_rag, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&ctl->s_full[i], 1);
       mbar_init(&ctl->p_full[i], 128);
@@ -112,13 +116,26 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
     // ================================ TMA producer ==========================================
     setmaxnreg_dec<kRegsOther>();
     if (lane == 0) {
-      uint32_t kvp = 0;
+      uint32_t kvp = 0, n_rag = 0;
       int seg = 0;
       bool q_armed = false;
+      constexpr bool dev_len = DEVLEN;
+      const int L_eff = DEVLEN ? spx_prefix_len(a) : p.L;
+      const int tph_eff = DEVLEN ? (L_eff + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
       for (int u = unit_lo; u < unit_hi && ok;) {
         const int prob = u / p.UPP;
         const int tile_lo = u - prob * p.UPP;
-        const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+        const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+        SpxSeg sg;
+        if (DEVLEN) {
+          sg = spx_segment(p, tile_lo, n_units, tph_eff);
+        } else {
+          sg.n_pref = n_units;                 // (the tree tile, if any, is simply the last of the run)
+          sg.has_tree = 0;
+          sg.n = n_units;
+        }
+        u += n_units;
+        if (DEVLEN && sg.n == 0) continue;     // nothing of this run exists at the device-side length
         const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
         if (seg > 0) ok = mbar_wait(&ctl->q_free, (seg - 1) & 1, abort_flag);
         if (!ok) break;
@@ -128,21 +145,43 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           for (int ds = 0; ds < DS; ++ds)
             tma_load_3d(Qs + (mt * DS + ds) * kSubTileBytes, &maps.q, &ctl->q_full, ds * 64, g * p.G,
                         (rblk * n_mt + mt) * (128 / p.G));
-        for (int tile = tile_lo; tile < tile_hi && ok; ++tile) {
+        for (int j = 0; j < sg.n && ok; ++j) {
+          const int tile = DEVLEN ? spx_seg_tile(p, sg, tile_lo, j) : tile_lo + j;
           const bool is_tree = tile == p.TPH;
+          const int nk = is_tree ? SPX_TILE_KEYS : L_eff - tile * SPX_TILE_KEYS;
           for (int which = 0; which < 2; ++which) {
             const int stage = kvp % NS;
             ok = mbar_wait(&ctl->kv_empty[stage], ((kvp / NS) & 1) ^ 1, abort_flag);
             if (!ok) break;
-            mbar_arrive_expect_tx(&ctl->kv_full[stage], C::kStageBytes);
             const CUtensorMap* m = is_tree ? (which ? &maps.vt : &maps.kt) : (which ? &maps.vp : &maps.kp);
-            for (int ds = 0; ds < DS; ++ds)
-              tma_load_3d(ring + stage * C::kStageBytes + ds * kSubTileBytes, m, &ctl->kv_full[stage], ds * 64, g,
-                          is_tree ? 0 : tile * SPX_TILE_KEYS);
+            unsigned char* dst = ring + stage * C::kStageBytes;
+            if (which == 1 && dev_len && nk < SPX_TILE_KEYS) {
+              // Device-side length: the tensor map spans the whole capacity, so the rows of this V tile
+              // past the length hold whatever the cache holds (their probabilities are zero, but zero
+              // times a NaN is a NaN).  The tile lands on a barrier of its own, its tail rows are
+              // cleared (a row of a 64-column block is 128 bytes whatever the swizzle), and only then
+              // is the stage handed to the MMA issuer.
+              mbar_arrive_expect_tx(&ctl->v_rag, C::kStageBytes);
+              for (int ds = 0; ds < DS; ++ds)
+                tma_load_3d(dst + ds * kSubTileBytes, m, &ctl->v_rag, ds * 64, g, tile * SPX_TILE_KEYS);
+              ok = mbar_wait(&ctl->v_rag, n_rag & 1, abort_flag);
+              if (!ok) break;
+              ++n_rag;
+              for (int ds = 0; ds < DS; ++ds) {
+                uint4* tail = reinterpret_cast<uint4*>(dst + ds * kSubTileBytes + nk * 128);
+                for (int i = 0; i < (SPX_TILE_KEYS - nk) * 8; ++i) tail[i] = make_uint4(0u, 0u, 0u, 0u);
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              mbar_arrive(&ctl->kv_full[stage]);
+            } else {
+              mbar_arrive_expect_tx(&ctl->kv_full[stage], C::kStageBytes);
+              for (int ds = 0; ds < DS; ++ds)
+                tma_load_3d(dst + ds * kSubTileBytes, m, &ctl->kv_full[stage], ds * 64, g,
+                            is_tree ? 0 : tile * SPX_TILE_KEYS);
+            }
             ++kvp;
           }
         }
-        u += tile_hi - tile_lo;
         ++seg;
       }
       if (!ok) {
@@ -216,11 +255,14 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           for (int kk = 1; kk < SPX_TILE_KEYS / 16; ++kk) mma_ts2(d, pa + kk * 8, vb + kk * 128, hi, idesc_o, 1u);
         };
 
+        const int tph_eff = DEVLEN ? (spx_prefix_len(a) + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
         for (int u = unit_lo; u < unit_hi && ok;) {
           const int prob = u / p.UPP;
           const int tile_lo = u - prob * p.UPP;
-          const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
-          const int n = tile_hi - tile_lo;
+          const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+          const int n = DEVLEN ? spx_segment(p, tile_lo, n_units, tph_eff).n : n_units;
+          u += n_units;
+          if (DEVLEN && n == 0) continue;
           ok = mbar_wait(&ctl->q_full, seg & 1, abort_flag);
           if (!ok) break;
           {
@@ -262,7 +304,6 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             ++it;
           }
           if (ok) mma_commit(&ctl->q_free);
-          u += n;
           ++seg;
         }
         // drain: all MMAs issued so far must have completed before tensor memory is released
@@ -285,19 +326,37 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
         const float scale2 = p.scale2;
         uint32_t it = 0;
         int seg = 0;
+        const int L_eff = DEVLEN ? spx_prefix_len(a) : p.L;
+        const int tph_eff = DEVLEN ? (L_eff + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
         for (int u = unit_lo; u < unit_hi && ok;) {
           const int prob = u / p.UPP;
           const int tile_lo = u - prob * p.UPP;
-          const int tile_hi = min(p.UPP, tile_lo + (unit_hi - u));
+          const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+          SpxSeg sg;
+          if (DEVLEN) sg = spx_segment(p, tile_lo, n_units, tph_eff);
+          const int n_seg = DEVLEN ? sg.n : n_units;
           const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
           const int r = rblk * p.RB + rr;
           const bool valid = r < p.rows;
+          if (DEVLEN && n_seg == 0) {
+            // No tile of this run exists at the device-side length: its slot gets the neutral partial
+            // (weight zero in the merge), and no barrier of the pipeline is touched.
+            const int slot = cta + prob;
+            float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
+            for (int q4 = 0; q4 < D / 4; ++q4)
+              *reinterpret_cast<float4*>(po + ((long long)q4 * p.RB + rr) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+            a.ws[p.off_part_m + (long long)slot * p.RB + rr] = -1e30f;      // finite: see the merge
+            a.ws[p.off_part_l + (long long)slot * p.RB + rr] = 0.f;
+            u += n_units;
+            continue;
+          }
           const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
           float m_used = -INFINITY, l = 0.f;
 
-          for (int tile = tile_lo; tile < tile_hi; ++tile, ++it) {
+          for (int j = 0; j < n_seg; ++j, ++it) {
+            const int tile = DEVLEN ? spx_seg_tile(p, sg, tile_lo, j) : tile_lo + j;
             const bool is_tree = tile == p.TPH;
-            const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
+            const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, (DEVLEN ? L_eff : p.L) - tile * SPX_TILE_KEYS);
             const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
             ok = mbar_wait(&ctl->s_full[mt], it & 1, abort_flag);
             if (!ok) break;
@@ -343,7 +402,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             bool rescale = false;
             if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
               alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
-              rescale = tile > tile_lo;
+              rescale = j > 0;
               m_used = m_tile;
               l *= alpha;
             }
@@ -442,7 +501,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           }
           tc_fence_before();
           mbar_arrive(&ctl->o_free[mt]);
-          u += tile_hi - tile_lo;
+          u += n_units;
           ++seg;
         }
       }
@@ -489,12 +548,12 @@ bool encode_map(CUtensorMap* m, const void* ptr, int D, long long n1, long long 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, bool SCORE>
+template <int D, bool SCORE, bool DEVLEN>
 cudaError_t launch(const AttnArgs& a, const TcMaps& maps, cudaStream_t st) {
   static SpxOncePerDevice once;
-  const cudaError_t ec = spx_opt_in_smem(attn_tc_kernel<D, SCORE>, Cfg<D>::kSmemBytes, &once);
+  const cudaError_t ec = spx_opt_in_smem(attn_tc_kernel<D, SCORE, DEVLEN>, Cfg<D>::kSmemBytes, &once);
   if (ec != cudaSuccess) return ec;
-  attn_tc_kernel<D, SCORE><<<a.plan.n_cta, kThreads, Cfg<D>::kSmemBytes, st>>>(a, maps);
+  attn_tc_kernel<D, SCORE, DEVLEN><<<a.plan.n_cta, kThreads, Cfg<D>::kSmemBytes, st>>>(a, maps);
   return cudaGetLastError();
 }
 
@@ -516,10 +575,12 @@ cudaError_t spx_launch_attn_tc(const AttnArgs& a, cudaStream_t st, int* n_launch
   }
   if (!ok) return cudaErrorInvalidValue;
   cudaError_t e;
-  if (p.D == 128)
-    e = p.want_score ? launch<128, true>(a, maps, st) : launch<128, false>(a, maps, st);
+  if (a.L_dev)                                  // never with chunk sums
+    e = p.D == 128 ? launch<128, false, true>(a, maps, st) : launch<64, false, true>(a, maps, st);
+  else if (p.D == 128)
+    e = p.want_score ? launch<128, true, false>(a, maps, st) : launch<128, false, false>(a, maps, st);
   else
-    e = p.want_score ? launch<64, true>(a, maps, st) : launch<64, false>(a, maps, st);
+    e = p.want_score ? launch<64, true, false>(a, maps, st) : launch<64, false, false>(a, maps, st);
   *n_launches += 1;
   return e;
 }

@@ -68,6 +68,7 @@ struct Ctrl {
   uint64_t drain;
   uint64_t anc_ready;           // this CTA: the ancestor masks are in shared memory
   uint64_t q_land;              // this CTA: the first segment's Q rows have landed in the scratch (TMA)
+  uint64_t v_rag;               // this CTA: a V half whose tail rows must be cleared has landed (device-side length)
   uint64_t epi[2];              // this CTA: 8 arrivals, the two meeting points of a segment's epilogue
   unsigned long long anc[64];
   int parent[64];
@@ -102,6 +103,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 }
 __device__ __forceinline__ void arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Arrival that publishes the thread's earlier writes at cluster scope (used where plain stores, not TMA
+// or tensor-memory traffic, precede it).
+__device__ __forceinline__ void arrive_release_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr),
@@ -183,7 +189,9 @@ __device__ __forceinline__ void commit_pair(uint64_t* bar) {
 // SCORE: 0 no chunk sums; otherwise the class of the chunk size, so that each variant carries only the
 // code it runs (the loop of the exponentials is instruction-cache sensitive): 1 chunks of 32 keys,
 // 2 chunks of 64 or 128 keys, 3 chunks of fewer than 32 keys.
-template <int SCORE>
+// DEVLEN: the prefix length is read from device memory (a.L_dev) and may be shorter than the planned
+// capacity p.L; the instantiation without it carries none of that code.
+template <int SCORE, bool DEVLEN>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2Maps maps) {
   const AttnPlan& p = a.plan;
@@ -221,6 +229,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       mbar_init(&ctl->drain, 2);
       mbar_init(&ctl->anc_ready, 1);
       mbar_init(&ctl->q_land, 1);
+      mbar_init(&ctl->v_rag, 1);
       ctl->abort_flag = 0;
     }
     fence_mbar_init();
@@ -243,7 +252,10 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
   // producer leaves alone until the first S MMA is done.  One thread fetches it with two TMA boxes
   // of 64 elements x G heads x 128/G nodes: exactly the stacked rows (G is a power of two), rows
   // past the tree zero-filled.
-  if (warp == kProducerWarp && lane == 0 && unit_lo < unit_hi) {
+  // (With a device-side prefix length the first segment may turn out to be empty; its Q rows then
+  // come by plain loads like those of every later segment.)
+  constexpr bool dev_len = DEVLEN;
+  if (warp == kProducerWarp && lane == 0 && unit_lo < unit_hi && !dev_len) {
     const int prob = unit_lo / p.UPP;
     const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
     const int t0 = (rblk * p.RB + (int)rank * 128) / p.G;
@@ -287,68 +299,164 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       uint32_t kp = 0, vp = 0;
       const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
       const uint32_t vfull0 = map_to_cta(smem_u32(&ctl->v_full[0]), 0);
-      // position in the line of units
-      struct Cursor {
-        int unit, tile, prob, g;
-      };
-      auto step = [&](Cursor& c) {
-        ++c.unit;
-        if (++c.tile == p.UPP) {
-          c.tile = 0;
-          ++c.prob;
-          c.g = c.prob / p.n_rblk;
+      if constexpr (!DEVLEN) {
+        // position in the line of units
+        struct Cursor {
+          int unit, tile, prob, g;
+        };
+        auto step = [&](Cursor& c) {
+          ++c.unit;
+          if (++c.tile == p.UPP) {
+            c.tile = 0;
+            ++c.prob;
+            c.g = c.prob / p.n_rblk;
+          }
+        };
+        // K half of a unit: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
+        auto load_k = [&](const Cursor& c) -> bool {
+          const int tile = c.tile, g = c.g;
+          const bool is_tree = tile == p.TPH;
+          const int stage = kp % kStages;
+          if (!wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag)) return false;
+          const uint32_t bar = kfull0 + stage * 8;
+          const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+          const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
+          const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
+          arrive_expect_tx_cluster(bar, kStageBytes);
+          tma_load_3d_pair(dst, m, bar, 0, g, key0);
+          tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
+          ++kp;
+          return true;
+        };
+        // V half of a unit: value columns [64*rank, 64*rank+64) of all 128 keys
+        auto load_v = [&](const Cursor& c) -> bool {
+          const int tile = c.tile, g = c.g;
+          const bool is_tree = tile == p.TPH;
+          const int stage = vp % kStages;
+          if (!wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag)) return false;
+          const uint32_t bar = vfull0 + stage * 8;
+          const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
+          arrive_expect_tx_cluster(bar, kStageBytes);
+          tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
+          ++vp;
+          return true;
+        };
+        // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A full
+        // ring requested at once by every SM sits in the memory system's queues in no particular order,
+        // and tile 0 would arrive last as often as first.
+        Cursor ck;
+        ck.unit = unit_lo;
+        ck.prob = unit_lo / p.UPP;
+        ck.tile = unit_lo - ck.prob * p.UPP;
+        ck.g = ck.prob / p.n_rblk;
+        Cursor cv = ck;
+        for (int i = 0; i < 2 && ck.unit < unit_hi && ok; ++i) {
+          ok = load_k(ck);
+          step(ck);
+          if (ok) ok = load_v(cv);
+          step(cv);
         }
-      };
-      // K half of a unit: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
-      auto load_k = [&](const Cursor& c) -> bool {
-        const int tile = c.tile, g = c.g;
-        const bool is_tree = tile == p.TPH;
-        const int stage = kp % kStages;
-        if (!wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag)) return false;
-        const uint32_t bar = kfull0 + stage * 8;
-        const uint32_t dst = smem_u32(ring + stage * kStageBytes);
-        const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
-        const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
-        arrive_expect_tx_cluster(bar, kStageBytes);
-        tma_load_3d_pair(dst, m, bar, 0, g, key0);
-        tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
-        ++kp;
-        return true;
-      };
-      // V half of a unit: value columns [64*rank, 64*rank+64) of all 128 keys
-      auto load_v = [&](const Cursor& c) -> bool {
-        const int tile = c.tile, g = c.g;
-        const bool is_tree = tile == p.TPH;
-        const int stage = vp % kStages;
-        if (!wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag)) return false;
-        const uint32_t bar = vfull0 + stage * 8;
-        const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
-        arrive_expect_tx_cluster(bar, kStageBytes);
-        tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
-        ++vp;
-        return true;
-      };
-      // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A full
-      // ring requested at once by every SM sits in the memory system's queues in no particular order,
-      // and tile 0 would arrive last as often as first.
-      Cursor ck;
-      ck.unit = unit_lo;
-      ck.prob = unit_lo / p.UPP;
-      ck.tile = unit_lo - ck.prob * p.UPP;
-      ck.g = ck.prob / p.n_rblk;
-      Cursor cv = ck;
-      for (int i = 0; i < 2 && ck.unit < unit_hi && ok; ++i) {
-        ok = load_k(ck);
-        step(ck);
-        if (ok) ok = load_v(cv);
-        step(cv);
-      }
-      if (ok && unit_lo < unit_hi) ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
-      while (ok && ck.unit < unit_hi) {
-        ok = load_k(ck);
-        step(ck);
-        if (ok) ok = load_v(cv);
-        step(cv);
+        if (ok && unit_lo < unit_hi) ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
+        while (ok && ck.unit < unit_hi) {
+          ok = load_k(ck);
+          step(ck);
+          if (ok) ok = load_v(cv);
+          step(cv);
+        }
+      } else {
+        const int L_eff = spx_prefix_len(a);
+        const int tph_eff = (L_eff + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS;
+        uint32_t n_rag = 0;
+        // position in the line of units: the run of units inside one problem and the tile inside the run
+        struct Cursor {
+          int u, g, tile_lo, n_units, j;
+          SpxSeg sg;
+        };
+        auto enter = [&](Cursor& c) {                 // moves to the next run that has tiles to process
+          while (c.u < unit_hi) {
+            const int prob = c.u / p.UPP;
+            c.tile_lo = c.u - prob * p.UPP;
+            c.n_units = min(p.UPP - c.tile_lo, unit_hi - c.u);
+            c.sg = spx_segment(p, c.tile_lo, c.n_units, tph_eff);
+            c.g = prob / p.n_rblk;
+            c.j = 0;
+            if (c.sg.n > 0) return;
+            c.u += c.n_units;
+          }
+        };
+        auto step = [&](Cursor& c) {
+          if (++c.j == c.sg.n) {
+            c.u += c.n_units;
+            enter(c);
+          }
+        };
+        // K half of a unit: keys [64*rank, 64*rank+64) of the tile, two 64-column blocks
+        auto load_k = [&](const Cursor& c) -> bool {
+          const int tile = spx_seg_tile(p, c.sg, c.tile_lo, c.j), g = c.g;
+          const bool is_tree = tile == p.TPH;
+          const int stage = kp % kStages;
+          if (!wait_c(&ctl->k_empty[stage], ((kp / kStages) & 1) ^ 1, abort_flag)) return false;
+          const uint32_t bar = kfull0 + stage * 8;
+          const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+          const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
+          const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
+          arrive_expect_tx_cluster(bar, kStageBytes);
+          tma_load_3d_pair(dst, m, bar, 0, g, key0);
+          tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
+          ++kp;
+          return true;
+        };
+        // V half of a unit: value columns [64*rank, 64*rank+64) of all 128 keys
+        auto load_v = [&](const Cursor& c) -> bool {
+          const int tile = spx_seg_tile(p, c.sg, c.tile_lo, c.j), g = c.g;
+          const bool is_tree = tile == p.TPH;
+          const int stage = vp % kStages;
+          if (!wait_c(&ctl->v_empty[stage], ((vp / kStages) & 1) ^ 1, abort_flag)) return false;
+          const uint32_t bar = vfull0 + stage * 8;
+          unsigned char* dstp = ring + (kStages + stage) * kStageBytes;
+          const int nk = is_tree ? SPX_TILE_KEYS : L_eff - tile * SPX_TILE_KEYS;
+          if (dev_len && nk < SPX_TILE_KEYS) {
+            // Device-side length: the tensor map spans the whole capacity, so the rows of this tile past the
+            // length hold whatever the cache holds (their probabilities are zero, but zero times a NaN is
+            // a NaN).  The half lands on a barrier of this CTA, its tail rows are cleared (a row is 128
+            // bytes whatever the swizzle), and only then is the stage handed to the MMA issuer.
+            mbar_arrive_expect_tx(&ctl->v_rag, kStageBytes);
+            tma_load_3d(dstp, &maps.vp, &ctl->v_rag, 64 * rank, g, tile * SPX_TILE_KEYS);
+            if (!mbar_wait(&ctl->v_rag, n_rag & 1, abort_flag)) return false;
+            ++n_rag;
+            uint4* tail = reinterpret_cast<uint4*>(dstp + nk * 128);
+            for (int i = 0; i < (SPX_TILE_KEYS - nk) * 8; ++i) tail[i] = make_uint4(0u, 0u, 0u, 0u);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            arrive_release_cluster(bar);
+          } else {
+            arrive_expect_tx_cluster(bar, kStageBytes);
+            tma_load_3d_pair(smem_u32(dstp), is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g,
+                             is_tree ? 0 : tile * SPX_TILE_KEYS);
+          }
+          ++vp;
+          return true;
+        };
+        // Start-up: only two tiles are requested until the first S MMA has consumed K tile 0.  A full
+        // ring requested at once by every SM sits in the memory system's queues in no particular order,
+        // and tile 0 would arrive last as often as first.
+        Cursor ck;
+        ck.u = unit_lo;
+        enter(ck);
+        Cursor cv = ck;
+        const bool any = ck.u < unit_hi;
+        for (int i = 0; i < 2 && ck.u < unit_hi && ok; ++i) {
+          ok = load_k(ck);
+          step(ck);
+          if (ok) ok = load_v(cv);
+          step(cv);
+        }
+        if (ok && any) ok = wait_c(&ctl->k_empty[0], 0, abort_flag);
+        while (ok && ck.u < unit_hi) {
+          ok = load_k(ck);
+          step(ck);
+          if (ok) ok = load_v(cv);
+          step(cv);
+        }
       }
     }
   } else {
@@ -397,10 +505,14 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const uint32_t ring_lo = desc_lo(smem_u32(ring), 16);
         uint32_t kc = 0, n_w[2] = {0, 0};          // n_w[w]: S tiles issued so far for warpgroup w
         int seg = 0;
+        const int tph_eff = DEVLEN ? (spx_prefix_len(a) + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
         for (int u = unit_lo; u < unit_hi && ok;) {
           const int prob = u / p.UPP;
           const int tile_lo = u - prob * p.UPP;
-          const int n = min(p.UPP - tile_lo, unit_hi - u);
+          const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+          const int n = DEVLEN ? spx_segment(p, tile_lo, n_units, tph_eff).n : n_units;
+          u += n_units;
+          if (DEVLEN && n == 0) continue;          // nothing of this run exists at the device-side length
           ok = wait_c(&ctl->q_ready, seg & 1, abort_flag);
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
@@ -420,7 +532,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             ++kc;
             ++n_w[w];
           }
-          u += n;
           ++seg;
         }
         commit_pair(&ctl->drain);
@@ -434,10 +545,14 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
         const uint32_t ring_lo = desc_lo(smem_u32(ring + kStages * kStageBytes), 16);
         uint32_t vc = 0;                           // V tiles consumed = PVs issued
         int seg = 0;
+        const int tph_eff = DEVLEN ? (spx_prefix_len(a) + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
         for (int u = unit_lo; u < unit_hi && ok;) {
           const int prob = u / p.UPP;
           const int tile_lo = u - prob * p.UPP;
-          const int n = min(p.UPP - tile_lo, unit_hi - u);
+          const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+          const int n = DEVLEN ? spx_segment(p, tile_lo, n_units, tph_eff).n : n_units;
+          u += n_units;
+          if (DEVLEN && n == 0) continue;
           ok = wait_c(&ctl->q_ready, seg & 1, abort_flag);      // every thread is done reading the previous O
           for (int j = 0; j < n && ok; ++j) {
             const int w = j & 1;
@@ -457,7 +572,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             if (j == n - 1) commit_pair(&ctl->o_done);
             ++vc;
           }
-          u += n;
           ++seg;
         }
         commit_pair(&ctl->drain);
@@ -485,19 +599,42 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
       uint32_t n_other = 0;      // tiles of the other warpgroup whose maxima this one has consumed
       uint32_t n_oth = 0;        // tiles the other warpgroup had been given before the current segment
       int seg = 0;
+      bool anc_seen = false;
+      const int L_eff = DEVLEN ? spx_prefix_len(a) : p.L;
+      const int tph_eff = DEVLEN ? (L_eff + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS : p.TPH;
       for (int u = unit_lo; u < unit_hi && ok;) {
         const int prob = u / p.UPP;
         const int tile_lo = u - prob * p.UPP;
-        const int n = min(p.UPP - tile_lo, unit_hi - u);
+        const int n_units = min(p.UPP - tile_lo, unit_hi - u);
+        SpxSeg sg;
+        if (DEVLEN) sg = spx_segment(p, tile_lo, n_units, tph_eff);
+        const int n = DEVLEN ? sg.n : n_units;
         const int g = prob / p.n_rblk, rblk = prob - g * p.n_rblk;
         const int r = rblk * p.RB + rr;
         const bool valid = r < p.rows;
         const int t_node = valid ? r / p.G : 0;
+        if (DEVLEN && n == 0) {
+          // No tile of this run exists at the device-side length: its slot gets the neutral partial
+          // (weight zero in the merge), and no barrier of the pipeline is touched.
+          const int slot = cl + prob;
+          if (valid) {
+            float* po = a.ws + p.off_part_o + (long long)slot * (D / 4) * p.RB * 4;
+#pragma unroll 4
+            for (int q4 = 0; q4 < 16; ++q4)
+              *reinterpret_cast<float4*>(po + ((long long)(wg * 16 + q4) * p.RB + rr) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (wg == 0) {
+              a.ws[p.off_part_m + (long long)slot * p.RB + rr] = -1e30f;      // finite: see the merge
+              a.ws[p.off_part_l + (long long)slot * p.RB + rr] = 0.f;
+            }
+          }
+          u += n_units;
+          continue;
+        }
         // Q row of this thread -> tensor memory (warpgroup 0: first 64 elements, warpgroup 1: the rest)
         {
           uint32_t qv[32];
           const __nv_bfloat16* qbase = a.Q + (long long)(g * p.G) * a.q_sh + wg * 64;
-          if (seg == 0) {
+          if (seg == 0 && !dev_len) {
             // requested at kernel start (see above)
             const unsigned char* scratch = ring + (2 * kStages - 2) * kStageBytes + warp * 4096;
             ok = mbar_wait(&ctl->q_land, 0, abort_flag);
@@ -526,17 +663,18 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           tc_fence_before();
           warp_arrive_cluster(q_ready_l, lane);
         }
-        if (seg == 0) {
+        if (DEVLEN ? !anc_seen : seg == 0) {
           ok = mbar_wait(&ctl->anc_ready, 0, abort_flag);
           if (!ok) break;
+          anc_seen = true;
         }
         const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
 
         float m_loc = -INFINITY, l = 0.f;        // l is relative to m_loc
         for (int j = wg; j < n && ok; j += 2) {
-          const int tile = tile_lo + j;
+          const int tile = DEVLEN ? spx_seg_tile(p, sg, tile_lo, j) : tile_lo + j;
           const bool is_tree = tile == p.TPH;
-          const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, p.L - tile * SPX_TILE_KEYS);
+          const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, (DEVLEN ? L_eff : p.L) - tile * SPX_TILE_KEYS);
           const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
           ok = wait_c(&ctl->s_full[wg], n_mine & 1, abort_flag);
           if (!ok) break;
@@ -744,7 +882,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             a.ws[p.off_part_l + (long long)slot * p.RB + rr] = l + ctl->l_x[row_t];
           }
         }
-        u += n;
+        u += n_units;
         if (u < unit_hi) {
           warp_arrive(&ctl->epi[1], lane);               // l_x and m_row may be reused
           ok = mbar_wait(&ctl->epi[1], seg & 1, abort_flag);
@@ -808,10 +946,10 @@ bool encode_q_map(CUtensorMap* m, const void* ptr, int T, int Hq, int G, long lo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int SCORE>
+template <int SCORE, bool DEVLEN>
 cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
   static SpxOncePerDevice once;
-  const cudaError_t ec = spx_opt_in_smem(attn_tc2_kernel<SCORE>, kSmemBytes, &once);
+  const cudaError_t ec = spx_opt_in_smem(attn_tc2_kernel<SCORE, DEVLEN>, kSmemBytes, &once);
   if (ec != cudaSuccess) return ec;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * a.plan.n_cta);
@@ -827,7 +965,7 @@ cudaError_t launch2(const AttnArgs& a, const Tc2Maps& maps, cudaStream_t st) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, attn_tc2_kernel<SCORE>, a, maps);
+  return cudaLaunchKernelEx(&cfg, attn_tc2_kernel<SCORE, DEVLEN>, a, maps);
 }
 
 }  // namespace
@@ -848,10 +986,11 @@ cudaError_t spx_launch_attn_tc2(const AttnArgs& a, cudaStream_t st, int* n_launc
   }
   ok = ok && encode_q_map(&maps.q, a.Q, p.T, p.Hq, p.G, a.q_st, a.q_sh);
   if (!ok) return cudaErrorInvalidValue;
-  const cudaError_t e = !p.want_score ? launch2<0>(a, maps, st)
-                        : p.C == 32   ? launch2<1>(a, maps, st)
-                        : p.C > 32    ? launch2<2>(a, maps, st)
-                                      : launch2<3>(a, maps, st);
+  const cudaError_t e = a.L_dev       ? launch2<0, true>(a, maps, st)       // never with chunk sums
+                        : !p.want_score ? launch2<0, false>(a, maps, st)
+                        : p.C == 32   ? launch2<1, false>(a, maps, st)
+                        : p.C > 32    ? launch2<2, false>(a, maps, st)
+                                      : launch2<3, false>(a, maps, st);
   *n_launches += 1;
   return e;
 }

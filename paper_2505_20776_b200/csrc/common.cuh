@@ -17,6 +17,7 @@ struct AttnArgs {
   const __nv_bfloat16* Kt;
   const __nv_bfloat16* Vt;
   const int32_t* parent;
+  const int32_t* L_dev;     // device-side prefix length (<= plan.L, the planned capacity), or null: the length is plan.L
   __nv_bfloat16* O;
   float* lse;
   float* chunk_score;
@@ -28,6 +29,14 @@ struct AttnArgs {
 
 __device__ __forceinline__ void spx_raise(int32_t* status, int code) {
   if (status) atomicOr(status, 1 << code);
+}
+
+// Prefix length of this call.  A device-side length is read from global memory, so only after the
+// kernel's dependency wait; it is clamped to [0, planned capacity].
+__device__ __forceinline__ int spx_prefix_len(const AttnArgs& a) {
+  if (!a.L_dev) return a.plan.L;
+  const int v = *reinterpret_cast<const volatile int32_t*>(a.L_dev);
+  return v < 0 ? 0 : (v > a.plan.L ? a.plan.L : v);
 }
 
 // Ancestor-or-self bit masks of the draft tree: bit u of anc[t] is set iff u == t or u is a

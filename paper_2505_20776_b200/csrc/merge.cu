@@ -39,6 +39,8 @@ __device__ __forceinline__ void merge_batch(const float* __restrict__ pm, const 
   float Mb = M;
 #pragma unroll
   for (int k = 0; k < B; ++k) Mb = fmaxf(Mb, ms[k]);
+  // (A worker that found no key, because a device-side length was shorter than planned, leaves the
+  // neutral partial m = -1e30, l = 0, O = 0: finite, so that no difference of maxima is inf - inf.)
   const float carry = sm100::ex2_approx(M - Mb);    // 0 on the first batch (M = -inf)
   Z *= carry;
   acc0.x *= carry; acc0.y *= carry; acc0.z *= carry; acc0.w *= carry;

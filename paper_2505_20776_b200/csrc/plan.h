@@ -68,4 +68,26 @@ SPX_HD int spx_unit_owner(const AttnPlan& p, int u) {
   return u < big ? u / (p.q + 1) : p.rem + (u - big) / p.q;
 }
 
+// The part of a worker's unit range that lies inside one problem is a run of `n_units` units starting
+// at tile `tile_lo`.  When the prefix length is only known on the device (Ld <= L, the planned
+// capacity), just the first tph_eff = ceil(Ld/128) prefix tiles exist; the tree tile (unit TPH, the
+// last of the problem) always does.  n = n_pref + has_tree tiles are processed: tile_lo + j for
+// j < n_pref, then the tree tile.  With tph_eff == TPH this is the planned run itself.
+struct SpxSeg {
+  int n_pref, has_tree, n;
+};
+SPX_HD SpxSeg spx_segment(const AttnPlan& p, int tile_lo, int n_units, int tph_eff) {
+  SpxSeg s;
+  const int end = tile_lo + n_units;                 // exclusive, <= UPP
+  s.has_tree = end == p.UPP ? 1 : 0;
+  int pref_end = end - s.has_tree;                   // <= TPH
+  if (pref_end > tph_eff) pref_end = tph_eff;
+  s.n_pref = pref_end > tile_lo ? pref_end - tile_lo : 0;
+  s.n = s.n_pref + s.has_tree;
+  return s;
+}
+SPX_HD int spx_seg_tile(const AttnPlan& p, const SpxSeg& s, int tile_lo, int j) {
+  return j < s.n_pref ? tile_lo + j : p.TPH;
+}
+
 #endif  // SPECEXT_PLAN_H_
