@@ -353,8 +353,8 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
           const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
           float m_used = -INFINITY, l = 0.f;
 
-          for (int j = 0; j < n_seg; ++j, ++it) {
-            const int tile = DEVLEN ? spx_seg_tile(p, sg, tile_lo, j) : tile_lo + j;
+          for (int jt = 0; jt < n_seg; ++jt, ++it) {
+            const int tile = DEVLEN ? spx_seg_tile(p, sg, tile_lo, jt) : tile_lo + jt;
             const bool is_tree = tile == p.TPH;
             const int nkeys = is_tree ? p.T : min(SPX_TILE_KEYS, (DEVLEN ? L_eff : p.L) - tile * SPX_TILE_KEYS);
             const bool need_mask = is_tree || nkeys < SPX_TILE_KEYS;
@@ -402,7 +402,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             bool rescale = false;
             if (m_tile > m_used + kRescaleThreshold || m_used == -INFINITY) {
               alpha = (m_used == -INFINITY) ? 0.f : ex2_approx(m_used - m_tile);
-              rescale = j > 0;
+              rescale = jt > 0;
               m_used = m_tile;
               l *= alpha;
             }

@@ -130,10 +130,10 @@ __device__ __forceinline__ bool try_wait_cluster(uint64_t* bar, uint32_t parity,
 // TMA writes (complete_tx), so the default CTA-scope semantics of arrive and wait suffice; cluster-scope
 // release/acquire on every arrival was measurably slower.
 __device__ __forceinline__ bool wait_c(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (try_wait_cluster(bar, parity, 0u)) return true;
+  if (mbar_test_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
-    if (try_wait_cluster(bar, parity, 20000u)) return true;
+    if (mbar_try_wait(bar, parity)) return true;       // may suspend the thread for a while
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitLimitCycles) {
       *abort_flag = 1;
