@@ -21,6 +21,8 @@ What the path computes, with the passage each part follows:
   from the last layer of the most recent verification pass).
 * SelectChunks and UpdateDraftCache of Algorithm 1 (Appendix A): keep the top-k chunks and
   rewrite the draft model's KV cache to hold only those.
+* The prefill of the prompt (Section 3.1: FlashAttention for the prefill stage of target and draft
+  model): ordinary causal self-attention.
 
 Readings taken where the paper is silent (each is listed with its reason in the design notes):
 a tree node attends to itself and its ancestors; query head h reads KV head h // (Hq/Hkv); the
@@ -35,7 +37,9 @@ general tree equals masked attention as computed by torch's fp64 scaled_dot_prod
 lse equals torch.logsumexp; zero queries give mass len_c / (L + depth + 1); a rank-one
 construction with exactly representable logits gives closed-form masses and outputs; a hand-worked
 rational example (tests/golden); select equals a brute-force sort; gather equals index
-arithmetic.  No function here is unpinned.
+arithmetic; the prefill equals torch's fp64 causal scaled_dot_product_attention, its first token
+returns V[0], and its block b equals verify_attn with the earlier tokens as prefix and the block as a
+chain tree.  No function here is unpinned.
 """
 from __future__ import annotations
 
@@ -162,6 +166,41 @@ def attn_split_merge(Q, K_prefix, V_prefix, K_tree, V_tree, parent, bounds: Sequ
         acc = sum(o * np.exp(m - M)[:, None] for m, o in zip(ms, os_))
         O[:, h, :] = acc / Z[:, None]
         lse[h, :] = M + np.log(Z)
+    return O, lse
+
+
+def prefill_attn(Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: Optional[float] = None,
+                 rows: Optional[Sequence[int]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Causal self-attention of the prompt (the prefill that Section 3.1 runs with FlashAttention).
+
+    Q [L][Hq][D], K, V [L][Hkv][D].  Token i attends to tokens 0..i (itself included), query head
+    h reads KV head h // (Hq/Hkv).  Plain definition, one query row at a time: the masked score
+    vector of the row is materialised, normalised once and multiplied with V.  `rows` restricts
+    the computation to those token positions (outputs are then indexed by position in `rows`),
+    which is how a long prompt is spot-checked.
+    Returns (O [n_rows][Hq][D], lse [Hq][n_rows]), natural logarithm, scale included.
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    L, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    assert K.shape == V.shape == (L, Hkv, D) and Hq % Hkv == 0
+    G = Hq // Hkv
+    scale = 1.0 / np.sqrt(D) if scale is None else float(scale)
+    rows = list(range(L)) if rows is None else [int(r) for r in rows]
+    O = np.zeros((len(rows), Hq, D))
+    lse = np.zeros((Hq, len(rows)))
+    for n, i in enumerate(rows):
+        assert 0 <= i < L
+        for h in range(Hq):
+            g = h // G
+            s = scale * (K[: i + 1, g, :] @ Q[i, h, :])          # visible keys only: 0..i
+            m = s.max()
+            p = np.exp(s - m)
+            Z = p.sum()
+            O[n, h, :] = (p / Z) @ V[: i + 1, g, :]
+            lse[h, n] = m + np.log(Z)
     return O, lse
 
 
