@@ -395,10 +395,22 @@ def main():
                 api.specext_draft_attn(d_dr, tdr["Q"], hp.K_compact[0], hp.V_compact[0], hp.n_tokens, tdr["K_tree"],
                                        tdr["V_tree"], pdr, O_dr, lse_dr, ws_dr, hp.status)
 
+        # prefill of a 16K-token prompt of the same layer shape (causal attention; K/V of layer 0, seeded Q)
+        wq = synth.Workload("prefill-q", w.n_q_heads, w.n_q_heads, w.head_dim, L, 1, w.chunk_size, 1, "chain", "needle",
+                            seed=seed + 9)
+        Q_pf = synth.make_layer(wq, device=dev)["K_prefix"]
+        O_pf = torch.empty_like(Q_pf)
+        lse_pf = torch.empty(w.n_q_heads, L, dtype=torch.float32, device=dev)
+
+        def prefill():
+            api.specext_prefill_attn(Q_pf, layers[0]["K_prefix"], layers[0]["V_prefix"], O_pf, lse_pf, hp.status)
+
         attn_us = part_us(attn_only, NL - 1)
         parts = {"scoreless_layer_us": attn_us, "score_layer_us": part_us(score_layers, n_sc),
                  "select_gather_us": part_us(retrieval_one_call, n_rt),
                  "select_then_gather_two_calls_us": part_us(retrieval_two_calls, n_rt),
+                 "prefill_16k_us": part_us(prefill, 1),
+                 "prefill_16k_flops": 4 * w.n_q_heads * w.head_dim * (L * (L + 1) // 2),
                  "draft_attn_us": part_us(draft_attn, n_rt),
                  "select_gather_then_draft_attn_us": part_us(retrieval_then_draft, n_rt),
                  "draft_attn_algorithmic_bytes": layer_work(wdr, pdr_np.tolist(), False)[0],
@@ -522,6 +534,8 @@ def main():
                           "achieved_gbs": nb_plain / (attn_us * 1e-6) / 1e9,
                           "achieved_tflops": fl_plain / (attn_us * 1e-6) / 1e12,
                           "t_hbm_us": ta_hbm, "t_tensor_us": ta_tc, "frac": max(ta_hbm, ta_tc) / attn_us}})
+        parts["prefill_16k_tflops"] = parts["prefill_16k_flops"] / (parts["prefill_16k_us"] * 1e-6) / 1e12
+        parts["prefill_16k_frac_of_tensor_peak"] = parts["prefill_16k_tflops"] / tf
         parts["draft_attn_t_hbm_us"] = parts["draft_attn_algorithmic_bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
         for o in others.values():
             th, tt = roof_times(o["algorithmic_bytes"], o["algorithmic_flops"], peaks, tf)

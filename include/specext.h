@@ -170,6 +170,29 @@ int specext_draft_attn(const specext_attn_desc* desc, const void* Q, const void*
                        size_t workspace_bytes, int32_t* device_status, void* cuda_stream);
 
 /*
+ * Prefill: causal self-attention over the L tokens of the prompt (Section 3.1, "Efficient
+ * Attention": the prefill stage of the target and of the draft model runs a tiled attention that
+ * never forms the L x L score matrix).  For every token i and query head h, with g = h / G:
+ *   s_j = scale * <Q[i,h], K[j,g]> for j <= i,  P = softmax(s),  O[i,h] = sum_j P_j V[j,g],
+ *   lse[h,i] = log sum_j exp(s_j).
+ * One kernel, no scratch memory: a block of 256/G consecutive tokens of one KV head (256 stacked
+ * query rows) is processed from its first to its last key tile by one pair of SMs, so nothing is
+ * split and nothing has to be merged.
+ *
+ *   desc  : n_q_heads, n_kv_heads, head_dim, softmax_scale and the strides q_stride_*, kv_stride_*,
+ *           o_stride_* are used; prefix_len is L >= 1, the number of prompt tokens; the other
+ *           fields are ignored.  head_dim must be 128 (UNSUPPORTED otherwise).
+ *   Q     : bf16 [L][Hq][D];  K, V : bf16 [>=L][Hkv][D], same strides;  O : bf16 [L][Hq][D];
+ *   lse   : fp32 [Hq][L], natural logarithm, softmax_scale included.
+ * Arithmetic as in specext_verify_attn.  The first retrieval after the prefill (Algorithm 1 runs
+ * SelectChunks / UpdateDraftCache before the first Draft) takes its scores from one
+ * specext_verify_attn call of the last layer with the last prompt token as a single tree node
+ * (n_tree = 1, parent = -1) over the prefix of the L - 1 tokens before it.
+ */
+int specext_prefill_attn(const specext_attn_desc* desc, const void* Q, const void* K, const void* V,
+                         void* O, float* lse, int32_t* device_status, void* cuda_stream);
+
+/*
  * SelectChunks followed by UpdateDraftCache (the two steps Algorithm 1 runs back to back when
  * doRetrieval is set) as ONE call: the same results, in idx, n_selected, K_out, V_out and
  * n_tokens_out, as specext_select_chunks(..., k, ...) followed by specext_gather_kv(...,

@@ -59,6 +59,8 @@ def bind(path: str) -> ctypes.CDLL:
                                     vp, vp]
     L.specext_draft_attn.restype = ctypes.c_int
     L.specext_draft_attn.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9 + [vp, sz, vp, vp]
+    L.specext_prefill_attn.restype = ctypes.c_int
+    L.specext_prefill_attn.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 7
     L.specext_select_gather.restype = ctypes.c_int
     L.specext_select_gather.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, i32, i64, i64, i64,
                                         vp, vp, vp, vp, vp, vp, vp]
@@ -161,6 +163,29 @@ def specext_draft_attn(desc: AttnDesc, Q: torch.Tensor, K_cache: torch.Tensor, V
                                   _ptr(K_tree), _ptr(V_tree), _ptr(parent), _ptr(O), _ptr(lse), _ptr(workspace),
                                   workspace.numel() * workspace.element_size(), _ptr(device_status), _stream())
     _check(rc, "specext_draft_attn")
+
+
+def specext_prefill_attn(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, O: torch.Tensor, lse: torch.Tensor,
+                         device_status: torch.Tensor, softmax_scale: float = 0.0) -> None:
+    """Enqueues the prefill (causal self-attention) of a prompt: Q, O [L][Hq][128], K, V [L][Hkv][128], lse [Hq][L]."""
+    for t, n in ((Q, "Q"), (K, "K"), (V, "V"), (O, "O")):
+        _bf16_3d(t, n)
+    if K.stride() != V.stride() or lse.dtype != torch.float32 or device_status.dtype != torch.int32:
+        raise ValueError("K and V must share strides; lse must be fp32 and device_status int32")
+    L, Hq, D = Q.shape
+    if K.shape[0] < L or O.shape != Q.shape or lse.numel() < Hq * L or not lse.is_contiguous():
+        raise ValueError("shapes: K, V [>=L][Hkv][D], O like Q, lse contiguous [Hq][L]")
+    d = AttnDesc()
+    d.n_q_heads, d.n_kv_heads, d.head_dim = Hq, K.shape[1], D
+    d.prefix_len, d.n_tree, d.chunk_size = L, 1, 32
+    d.softmax_scale, d.want_chunk_score = float(softmax_scale), 0
+    d.q_stride_t, d.q_stride_h = Q.stride(0), Q.stride(1)
+    d.kv_stride_l, d.kv_stride_h = K.stride(0), K.stride(1)
+    d.tkv_stride_t, d.tkv_stride_h = K.stride(0), K.stride(1)
+    d.o_stride_t, d.o_stride_h = O.stride(0), O.stride(1)
+    rc = lib().specext_prefill_attn(ctypes.byref(d), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(lse),
+                                    _ptr(device_status), _stream())
+    _check(rc, "specext_prefill_attn")
 
 
 STATIC_SCRATCH_BYTES = 32 << 20

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_PATH = os.path.join(HERE, "libspecext.so")
 TESTING_LIB_PATH = os.path.join(HERE, "libspecext_testing.so")
-SOURCES = ["api.cu", "attn_tc2.cu", "attn_tc.cu", "merge.cu", "retrieval.cu"]
+SOURCES = ["api.cu", "attn_tc2.cu", "attn_tc.cu", "prefill_tc2.cu", "merge.cu", "retrieval.cu"]
 TESTING_SOURCES = SOURCES + ["attn_simt.cu", "testing.cu"]
 
 

@@ -11,6 +11,10 @@ cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int 
                               long long s_layer, long long s_l, long long s_h, const int32_t* idx,
                               const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
                               int32_t* n_tokens_out, int32_t* status, cudaStream_t st);
+cudaError_t spx_launch_prefill_tc2(const void* Q, const void* K, const void* V, void* O, float* lse, int L, int Hq,
+                                   int Hkv, float scale2, long long q_st, long long q_sh, long long kv_sl,
+                                   long long kv_sh, long long o_st, long long o_sh, int n_sm, int32_t* status,
+                                   cudaStream_t st);
 bool spx_select_gather_fusable(int NC, int k);
 cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* dK, const void* dV, int n_layers,
                                      int H, int D, int L, int C, long long s_layer, long long s_l, long long s_h,
@@ -247,6 +251,35 @@ int specext_draft_attn(const specext_attn_desc* desc, const void* Q, const void*
   if (!n_tokens) return SPECEXT_ERR_INVALID_ARG;
   return run_attn(desc, Q, K_cache, V_cache, K_tree, V_tree, parent, n_tokens, O, lse, nullptr, workspace,
                   workspace_bytes, device_status, cuda_stream);
+}
+
+int specext_prefill_attn(const specext_attn_desc* desc, const void* Q, const void* K, const void* V, void* O,
+                         float* lse, int32_t* device_status, void* cuda_stream) {
+  if (!desc || !Q || !K || !V || !O || !lse) return SPECEXT_ERR_INVALID_ARG;
+  if (desc->n_q_heads < 1 || desc->n_kv_heads < 1 || desc->n_q_heads % desc->n_kv_heads != 0)
+    return SPECEXT_ERR_INVALID_ARG;
+  if (desc->prefix_len < 1 || desc->prefix_len > (1 << 24)) return SPECEXT_ERR_INVALID_ARG;
+  if (!(desc->softmax_scale >= 0.f) || !std::isfinite(desc->softmax_scale)) return SPECEXT_ERR_INVALID_ARG;
+  const int G = desc->n_q_heads / desc->n_kv_heads;
+  if (desc->head_dim != 128 || !is_pow2(G) || G > 256) return SPECEXT_ERR_UNSUPPORTED;
+  const long long strides[6] = {desc->q_stride_t, desc->q_stride_h, desc->kv_stride_l, desc->kv_stride_h,
+                                desc->o_stride_t, desc->o_stride_h};
+  for (long long s : strides)
+    if (s < desc->head_dim || (s & 7) != 0) return SPECEXT_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || (reinterpret_cast<uintptr_t>(lse) & 3u) != 0)
+    return SPECEXT_ERR_INVALID_ARG;
+  const float scale = desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / std::sqrt((float)desc->head_dim);
+  const cudaError_t e = spx_launch_prefill_tc2(Q, K, V, O, lse, desc->prefix_len, desc->n_q_heads, desc->n_kv_heads,
+                                               scale * 1.44269504088896340736f, desc->q_stride_t, desc->q_stride_h,
+                                               desc->kv_stride_l, desc->kv_stride_h, desc->o_stride_t,
+                                               desc->o_stride_h, sm_count(), device_status,
+                                               static_cast<cudaStream_t>(cuda_stream));
+  g_launches.fetch_add(1);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return SPECEXT_ERR_CUDA;
+  }
+  return SPECEXT_OK;
 }
 
 int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void* Q,

@@ -29,9 +29,10 @@
 // allocation and the start-up cluster barrier run while the kernel before it in the stream finishes;
 // global memory is touched only after griddepcontrol.wait.
 #include "common.cuh"
-#include "sm100.cuh"
+#include "pair.cuh"
 
 using namespace sm100;
+using namespace pair;
 
 struct Tc2Maps {
   CUtensorMap kp, vp, kt, vt;
@@ -78,113 +79,6 @@ struct Ctrl {
   int abort_flag;
 };
 static_assert(sizeof(Ctrl) <= 3072, "control block too large");
-
-__device__ __forceinline__ uint32_t cluster_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void cluster_arrive() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void cluster_wait() {
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Execution barrier only (no ordering of global memory): an arrival does not wait for the thread's
-// outstanding stores.
-__device__ __forceinline__ void cluster_sync_relaxed() {
-  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// Arrival that publishes the thread's earlier writes at cluster scope (used where plain stores, not TMA
-// or tensor-memory traffic, precede it).
-__device__ __forceinline__ void arrive_release_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void arrive_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr),
-               "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool try_wait_cluster(uint64_t* bar, uint32_t parity, uint32_t ns) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait on a barrier of this CTA whose arrivals may come from the peer CTA or from the pair's
-// tensor pipe.  What such a barrier orders is tensor-memory traffic (fenced with tcgen05.fence) and
-// TMA writes (complete_tx), so the default CTA-scope semantics of arrive and wait suffice; cluster-scope
-// release/acquire on every arrival was measurably slower.
-__device__ __forceinline__ bool wait_c(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_test_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;       // may suspend the thread for a while
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitCycles) {
-      *abort_flag = 1;
-      return false;
-    }
-  }
-}
-// One arrival for the whole warp: every lane has finished (and fenced) its own work; the warp
-// barrier orders those lanes before lane 0, whose release makes the warp's work visible.
-__device__ __forceinline__ void warp_arrive_cluster(uint32_t cluster_addr, int lane) {
-  __syncwarp();
-  if (lane == 0) arrive_cluster(cluster_addr);
-}
-__device__ __forceinline__ void warp_arrive(uint64_t* bar, int lane) {
-  __syncwarp();
-  if (lane == 0) mbar_arrive(bar);
-}
-// 3-D tiled load into this CTA's shared memory; the completion barrier may be the peer CTA's.
-__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster_addr,
-                                                 int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
-      "%5}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
-}
-// Asks for a tile to be brought into L2; needs no barrier and no shared memory.
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
-               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(c0), "r"(c1), "r"(c2)
-               : "memory");
-}
-// D[tmem, both CTAs] (+)= A[tmem, own rows of each CTA] * B[smem halves of both CTAs]
-__device__ __forceinline__ void mma_ts_pair(uint32_t d, uint32_t a, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                            uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-      ::"r"(d), "r"(a), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// One arrival on the barrier at this offset in both CTAs once all MMAs issued so far are complete.
-__device__ __forceinline__ void commit_pair(uint64_t* bar) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(smem_u32(bar)), "h"((uint16_t)3)
-      : "memory");
-}
-
 
 // SCORE: 0 no chunk sums; otherwise the class of the chunk size, so that each variant carries only the
 // code it runs (the loop of the exponentials is instruction-cache sensitive): 1 chunks of 32 keys,

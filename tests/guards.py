@@ -16,6 +16,17 @@ BAND_BYTES = 4096
 PATTERN = 0xA5
 
 
+class GuardedAlloc:
+    """Allocator of guarded device tensors; check() verifies every band handed out so far."""
+
+    def __init__(self, device):
+        self.device = torch.device(device)
+        self._bands: List[Tuple[str, torch.Tensor]] = []
+
+    _alloc = None           # filled in below (shared with GuardedHotPath)
+    check = None
+
+
 class GuardedHotPath(HotPath):
     """HotPath whose buffers (outputs, status words, indices, compact cache, workspace) are guarded."""
 
@@ -39,3 +50,8 @@ class GuardedHotPath(HotPath):
         for name, band in self._bands:
             bad = (band != PATTERN).nonzero()
             assert bad.numel() == 0, f"guard band {name} overwritten at byte offsets {bad[:8].flatten().tolist()}"
+
+
+GuardedAlloc._alloc = GuardedHotPath._alloc
+GuardedAlloc.alloc = GuardedHotPath._alloc
+GuardedAlloc.check = GuardedHotPath.check
