@@ -29,35 +29,37 @@ constexpr int kKeyCache = 2048;            // ranking keys kept in shared memory
 
 template <int NT>
 struct SelectSmem {
-  uint32_t hist[256];
-  uint32_t s_prefix, s_need;
-  uint32_t warp_tot[2][NT / 32];
-  uint32_t carry[2];
+  uint32_t hist[4][256];                   // one histogram per radix pass: cleared once, no barrier in between
+  uint32_t s_prefix[4], s_need[4];
+  uint32_t warp_eq[2][NT / 32], warp_keep[2][NT / 32];     // per batch of NT chunks, double-buffered
   uint32_t keys[kKeyCache];
 };
 
 // Selection by one block of NT threads: writes the keff = min(k, NC) kept chunk indices, ascending,
-// to idx_out (global or shared memory).  Every thread of the block must call it.
+// to idx_out (global or shared memory).  Every thread of the block must call it.  Two block barriers per
+// radix pass and two per batch of NT chunks in the emission.
 template <int NT>
 __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __restrict__ score, int NC, int L,
                                              int C, int keff, int32_t* idx_out) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NW = NT / 32;
   // one load and one division per chunk when the keys fit in shared memory
   const bool cached = NC <= kKeyCache;
   if (cached)
     for (int c = tid; c < NC; c += NT) sm.keys[c] = chunk_key(score, c, NC, L, C);
   auto key_of = [&](int c) -> uint32_t { return cached ? sm.keys[c] : chunk_key(score, c, NC, L, C); };
+  for (int i = tid; i < 4 * 256; i += NT) (&sm.hist[0][0])[i] = 0;
+  __syncthreads();
 
   // ---- radix select of the keff-th largest key --------------------------------------------
   uint32_t prefix = 0, need = keff;        // `need` keys still to take among those matching prefix
+#pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    if (tid < 256) sm.hist[tid] = 0;
-    __syncthreads();
     for (int c = tid; c < NC; c += NT) {
       const uint32_t key = key_of(c);
-      if ((key & himask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255u], 1u);
+      if ((key & himask) == prefix) atomicAdd(&sm.hist[pass][(key >> shift) & 255u], 1u);
     }
     __syncthreads();
     if (warp == 0) {
@@ -65,7 +67,7 @@ __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __
       uint32_t local[8], tot = 0;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        local[i] = sm.hist[255 - (lane * 8 + i)];
+        local[i] = sm.hist[pass][255 - (lane * 8 + i)];
         tot += local[i];
       }
       uint32_t incl = tot;
@@ -79,61 +81,65 @@ __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           if (before < need && need <= before + local[i]) {
-            sm.s_prefix = prefix | ((uint32_t)(255 - (lane * 8 + i)) << shift);
-            sm.s_need = need - before;
+            sm.s_prefix[pass] = prefix | ((uint32_t)(255 - (lane * 8 + i)) << shift);
+            sm.s_need[pass] = need - before;
           }
           before += local[i];
         }
       }
     }
     __syncthreads();
-    prefix = sm.s_prefix;
-    need = sm.s_need;
-    __syncthreads();
+    prefix = sm.s_prefix[pass];
+    need = sm.s_need[pass];
   }
   const uint32_t theta = prefix;           // the keff-th largest key
   const uint32_t need_eq = need;           // how many keys equal to theta are kept (lowest indices)
 
   // ---- emit in ascending index order --------------------------------------------------------
-  if (tid == 0) sm.carry[0] = sm.carry[1] = 0;
-  __syncthreads();
-  for (int base = 0; base < NC; base += NT) {
+  uint32_t carry_eq = 0, carry_keep = 0;   // totals of the batches before this one (the same in every thread)
+  int buf = 0;
+  for (int base = 0; base < NC; base += NT, buf ^= 1) {
     const int c = base + tid;
     uint32_t key = 0;
-    bool in = c < NC;
+    const bool in = c < NC;
     if (in) key = key_of(c);
     const bool eq = in && key == theta;
     const bool gt = in && key > theta;
-    // exclusive count of `eq` before this chunk
     const uint32_t beq = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) sm.warp_tot[0][warp] = __popc(beq);
+    if (lane == 0) sm.warp_eq[buf][warp] = __popc(beq);
     __syncthreads();
-    uint32_t eq_before = sm.carry[0] + __popc(beq & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) eq_before += sm.warp_tot[0][w];
+    uint32_t eq_before = carry_eq + __popc(beq & ((1u << lane) - 1u)), eq_all = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const uint32_t x = sm.warp_eq[buf][w];
+      eq_all += x;
+      if (w < warp) eq_before += x;
+    }
     const bool keep = gt || (eq && eq_before < need_eq);
     const uint32_t bk = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) sm.warp_tot[1][warp] = __popc(bk);
+    if (lane == 0) sm.warp_keep[buf][warp] = __popc(bk);
     __syncthreads();
-    uint32_t pos = sm.carry[1] + __popc(bk & ((1u << lane) - 1u));
-    for (int w = 0; w < warp; ++w) pos += sm.warp_tot[1][w];
-    if (keep && pos < (uint32_t)keff) idx_out[pos] = c;
-    __syncthreads();
-    if (tid == NT - 1) {
-      sm.carry[0] = eq_before + (eq ? 1u : 0u);
-      sm.carry[1] = pos + (keep ? 1u : 0u);
+    uint32_t pos = carry_keep + __popc(bk & ((1u << lane) - 1u)), keep_all = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const uint32_t x = sm.warp_keep[buf][w];
+      keep_all += x;
+      if (w < warp) pos += x;
     }
-    __syncthreads();
+    if (keep && pos < (uint32_t)keff) idx_out[pos] = c;
+    carry_eq += eq_all;
+    carry_keep += keep_all;
   }
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ score, int NC, int L,
-                                                             int C, int k, int32_t* __restrict__ idx,
-                                                             int32_t* __restrict__ n_selected) {
-  __shared__ SelectSmem<kSelThreads> sm;
+template <int NT>
+__global__ void __launch_bounds__(NT) select_kernel(const float* __restrict__ score, int NC, int L, int C, int k,
+                                                    int32_t* __restrict__ idx, int32_t* __restrict__ n_selected) {
+  __shared__ SelectSmem<NT> sm;
   sm100::pdl_launch_dependents();
   sm100::pdl_wait();                       // the scores are complete
   const int keff = min(k, NC);
-  select_block<kSelThreads>(sm, score, NC, L, C, keff, idx);
+  select_block<NT>(sm, score, NC, L, C, keff, idx);
   if (threadIdx.x == 0) *n_selected = keff;
 }
 
@@ -163,7 +169,23 @@ __device__ __forceinline__ void gather_part(const GatherArgs& g, int i, int c, i
   const __nv_bfloat16* src = g.src[which] + (long long)layer * g.s_layer;
   __nv_bfloat16* dst = g.dst[which] + ((long long)layer * g.max_selected * g.C + (long long)i * g.C) * g.H * g.D;
   const int nvec = max(0, o_hi - o_lo) * vpt;
-  // four vectors per thread and round: all loads are issued before the first store
+  if (g.s_h == g.D && g.s_l == (long long)g.H * g.D) {
+    // tokens are contiguous in the source as they are in the compact cache: a plain copy of one range,
+    // four vectors per thread and round, all loads issued before the first store
+    const uint4* sp = reinterpret_cast<const uint4*>(src + (long long)(c * g.C + o_lo) * g.s_l);
+    uint4* dp = reinterpret_cast<uint4*>(dst + (long long)o_lo * g.H * g.D);
+    for (int v0 = threadIdx.x; v0 < nvec; v0 += 4 * blockDim.x) {
+      uint4 x[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (v0 + q * (int)blockDim.x < nvec) x[q] = __ldg(sp + v0 + q * blockDim.x);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (v0 + q * (int)blockDim.x < nvec) dp[v0 + q * blockDim.x] = x[q];
+    }
+    return;
+  }
+  // strided source: four vectors per thread and round, all loads issued before the first store
   for (int v0 = threadIdx.x; v0 < nvec; v0 += 4 * blockDim.x) {
     uint4 x[4];
     long long off[4];
@@ -278,7 +300,10 @@ void fill_gather_args(GatherArgs& g, const void* dK, const void* dV, int n_layer
 cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
                               int32_t* n_selected, cudaStream_t st) {
   void* args[] = {&score_row, &NC, &L, &C, &k, &idx, &n_selected};
-  return launch_pdl(reinterpret_cast<const void*>(select_kernel), dim3(1), dim3(kSelThreads), args, st);
+  // few chunks: a small block, whose barriers are cheap; many: the widest one
+  if (NC <= 2048)
+    return launch_pdl(reinterpret_cast<const void*>(select_kernel<kFusedThreads>), dim3(1), dim3(kFusedThreads), args, st);
+  return launch_pdl(reinterpret_cast<const void*>(select_kernel<kSelThreads>), dim3(1), dim3(kSelThreads), args, st);
 }
 
 cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
