@@ -237,6 +237,7 @@ def _small(Hq, Hkv, D, L, T, C, k=4, tree="uniform", values="normal", seed=7):
     (2, 2, 64, 300, 64, 128),    # MHA (G = 1), maximum tree, maximum chunk size
     (64, 1, 128, 513, 5, 64),    # G = 64: 320 stacked rows -> two row blocks
     (16, 8, 128, 2048 + 77, 60, 8),
+    (8, 2, 128, 9000, 5, 1),     # 9000 chunks: the one-call retrieval takes its two-kernel route
 ])
 def test_edge_shapes(cuda_device, Hq, Hkv, D, L, T, C):
     w = _small(Hq, Hkv, D, L, T, C)
