@@ -24,7 +24,7 @@ What the path computes, with the passage each part follows:
 * The prefill of the prompt (Section 3.1: FlashAttention for the prefill stage of target and draft
   model): ordinary causal self-attention.
 
-Readings taken where the paper is silent (each is listed with its reason in the design notes):
+Readings taken where the paper is silent (each one is a stated choice of this build, not a fact of the paper):
 a tree node attends to itself and its ancestors; query head h reads KV head h // (Hq/Hkv); the
 softmax normaliser covers prefix and visible tree keys together; a chunk's exported score is the
 mean over all query heads of its summed probability ("mass"), and chunks are ranked by

@@ -191,6 +191,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     cluster_wait();                        // both CTAs' barriers exist
     if (lane == 0) {
       uint32_t kp = 0, vp = 0;
+      const uint64_t stream_once = policy_evict_first();
       const uint32_t kfull0 = map_to_cta(smem_u32(&ctl->k_full[0]), 0);      // leader's barriers
       const uint32_t vfull0 = map_to_cta(smem_u32(&ctl->v_full[0]), 0);
       if constexpr (!DEVLEN) {
@@ -217,8 +218,8 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
           const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
           arrive_expect_tx_cluster(bar, kStageBytes);
-          tma_load_3d_pair(dst, m, bar, 0, g, key0);
-          tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
+          tma_load_3d_pair_hint(dst, m, bar, 0, g, key0, stream_once);
+          tma_load_3d_pair_hint(dst + 8192, m, bar, 64, g, key0, stream_once);
           ++kp;
           return true;
         };
@@ -231,7 +232,8 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           const uint32_t bar = vfull0 + stage * 8;
           const uint32_t dst = smem_u32(ring + (kStages + stage) * kStageBytes);
           arrive_expect_tx_cluster(bar, kStageBytes);
-          tma_load_3d_pair(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS);
+          tma_load_3d_pair_hint(dst, is_tree ? &maps.vt : &maps.vp, bar, 64 * rank, g, is_tree ? 0 : tile * SPX_TILE_KEYS,
+                              stream_once);
           ++vp;
           return true;
         };
@@ -295,7 +297,7 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           const CUtensorMap* m = is_tree ? &maps.kt : &maps.kp;
           const int key0 = (is_tree ? 0 : tile * SPX_TILE_KEYS) + 64 * rank;
           arrive_expect_tx_cluster(bar, kStageBytes);
-          tma_load_3d_pair(dst, m, bar, 0, g, key0);
+          tma_load_3d_pair(dst, m, bar, 0, g, key0);       // (no eviction hint: a compact cache is read again at the next draft step)
           tma_load_3d_pair(dst + 8192, m, bar, 64, g, key0);
           ++kp;
           return true;
