@@ -211,12 +211,13 @@ def chunk_lengths(prefix_len: int, chunk_size: int) -> np.ndarray:
 
 
 def select_chunks(chunk_score_row: np.ndarray, prefix_len: int, chunk_size: int, k: int,
-                  key_dtype=np.float64) -> np.ndarray:
+                  key_dtype=np.float64, n_sink: int = 0, n_recent: int = 0) -> np.ndarray:
     """SelectChunks of Algorithm 1: indices of the top-k chunks, ascending.
 
     chunk_score_row [NC] holds summed probability per chunk; the ranking key is the chunk's
     average score, mass / len_c (Section 3.2.1).  Order: key descending, chunk index ascending
-    among equal keys; the first min(k, NC) are kept and returned sorted by index.  The key is
+    among equal keys; the first min(k, NC) are kept and returned sorted by index.  n_sink / n_recent
+    (an extension, default 0) force the earliest / latest chunks into the selection.  The key is
     formed in `key_dtype`: fp64 by default (the plain definition).  A test that hands the same
     fp32 score row to the oracle and to another implementation may ask for np.float32, so that
     the integer decision is taken in the same arithmetic on both sides.
@@ -224,9 +225,14 @@ def select_chunks(chunk_score_row: np.ndarray, prefix_len: int, chunk_size: int,
     score = np.asarray(chunk_score_row)
     NC = score.shape[0]
     assert NC == -(-prefix_len // chunk_size)
+    assert n_sink >= 0 and n_recent >= 0
     lens = chunk_lengths(prefix_len, chunk_size)
     key = (score.astype(key_dtype) / lens.astype(key_dtype)).astype(key_dtype)
-    order = sorted(range(NC), key=lambda c: (-float(key[c]), c))
+    # Optional extension (the paper's retrieval forces nothing: n_sink = n_recent = 0): the first n_sink
+    # and the last n_recent chunks are kept whatever their score, i.e. they rank above every other chunk
+    # (lower index first among themselves); the remaining places go to the best of the rest.
+    forced = [c < n_sink or c >= NC - n_recent for c in range(NC)]
+    order = sorted(range(NC), key=lambda c: (0 if forced[c] else 1, 0.0 if forced[c] else -float(key[c]), c))
     keep = order[:min(int(k), NC)]
     return np.array(sorted(keep), dtype=np.int32)
 

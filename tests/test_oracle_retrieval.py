@@ -96,3 +96,29 @@ def test_gather_equals_index_arithmetic():
     # nothing selected
     K, V, n = orc.gather_kv(dK, dV, [], L, C)
     assert n == 0 and K.shape[1] == 0
+
+
+def test_forced_sink_and_recent_chunks_by_set_definition():
+    """The extension: forced chunks first, then the best of the rest, against a definition by sets."""
+    rng = np.random.default_rng(9)
+    NC, C = 12, 4
+    L = NC * C - 1
+    lens = orc.chunk_lengths(L, C).astype(np.float64)
+    for trial in range(20):
+        score = rng.random(NC)
+        key = score / lens
+        for n_sink, n_recent, k in [(0, 0, 3), (1, 0, 3), (0, 2, 3), (2, 2, 6), (2, 2, 4), (3, 2, 4), (1, 1, 1),
+                                    (7, 7, 5), (0, 0, 12), (2, 1, 20)]:
+            forced = sorted(set(range(min(n_sink, NC))) | set(range(max(0, NC - n_recent), NC)))
+            keff = min(k, NC)
+            if len(forced) >= keff:
+                want = forced[:keff]                                     # sinks first: lowest indices
+            else:
+                rest = [c for c in range(NC) if c not in forced]
+                rest.sort(key=lambda c: (-key[c], c))
+                want = sorted(forced + rest[:keff - len(forced)])
+            got = orc.select_chunks(score, L, C, k, n_sink=n_sink, n_recent=n_recent)
+            assert got.tolist() == want, (n_sink, n_recent, k)
+    # nothing forced: exactly the plain selection
+    score = rng.random(NC)
+    np.testing.assert_array_equal(orc.select_chunks(score, L, C, 5), orc.select_chunks(score, L, C, 5, n_sink=0, n_recent=0))
