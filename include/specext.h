@@ -110,6 +110,10 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
  *   prefix_len, chunk_size : define n_chunks = ceil(L/C) (must equal the argument) and the
  *                 length len_c of the trailing chunk.  Any chunk_size >= 1 is accepted.
  *   k           : number of chunks to keep, >= 1; k_eff = min(k, n_chunks).
+ *   n_sink_chunks, n_recent_chunks : 0 and 0 for the paper's retrieval, which forces nothing.  As an
+ *                 extension the first n_sink_chunks and the last n_recent_chunks chunks are kept
+ *                 whatever their score: they rank above all others (lower index first among
+ *                 themselves) and the remaining places go to the best of the rest.
  *   idx         : int32 [min(k, n_chunks)] out, the kept chunk indices in ascending order.
  *   n_selected  : int32 [1] out (device), = k_eff.
  * Ranking key: chunk_score[row][c] / (float)len_c in fp32 (IEEE division); larger first, equal
@@ -117,8 +121,9 @@ int specext_verify_attn(const specext_attn_desc* desc, const void* Q, const void
  * n_chunks <= 65536.
  */
 int specext_select_chunks(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
-                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t* idx,
-                          int32_t* n_selected, int32_t* device_status, void* cuda_stream);
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t n_sink_chunks,
+                          int32_t n_recent_chunks, int32_t* idx, int32_t* n_selected,
+                          int32_t* device_status, void* cuda_stream);
 
 /*
  * UpdateDraftCache of Algorithm 1 (Appendix A; Section 3.2.1: the draft model keeps only the
@@ -195,13 +200,14 @@ int specext_prefill_attn(const specext_attn_desc* desc, const void* Q, const voi
 /*
  * SelectChunks followed by UpdateDraftCache (the two steps Algorithm 1 runs back to back when
  * doRetrieval is set) as ONE call: the same results, in idx, n_selected, K_out, V_out and
- * n_tokens_out, as specext_select_chunks(..., k, ...) followed by specext_gather_kv(...,
+ * n_tokens_out, as specext_select_chunks(..., k, n_sink_chunks, n_recent_chunks, ...) followed by specext_gather_kv(...,
  * max_selected = k, ...), argument for argument.  For n_chunks <= 8192 and k <= 1024 it is a single
  * kernel launch (every thread block repeats the deterministic selection and copies its share of the
  * kept chunks, so no block waits for another); larger sizes run the two kernels.
  */
 int specext_select_gather(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
-                          int32_t prefix_len, int32_t chunk_size, int32_t k, const void* draft_K,
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t n_sink_chunks,
+                          int32_t n_recent_chunks, const void* draft_K,
                           const void* draft_V, int32_t n_layers, int32_t n_kv_heads, int32_t head_dim,
                           int64_t stride_layer, int64_t stride_l, int64_t stride_h, int32_t* idx,
                           int32_t* n_selected, void* K_out, void* V_out, int32_t* n_tokens_out,

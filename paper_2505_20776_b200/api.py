@@ -53,7 +53,7 @@ def bind(path: str) -> ctypes.CDLL:
     L.specext_verify_attn_static_scratch.restype = ctypes.c_int
     L.specext_verify_attn_static_scratch.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 9 + [vp, vp]
     L.specext_select_chunks.restype = ctypes.c_int
-    L.specext_select_chunks.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+    L.specext_select_chunks.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     L.specext_gather_kv.restype = ctypes.c_int
     L.specext_gather_kv.argtypes = [vp, vp, i32, i32, i32, i32, i32, i64, i64, i64, vp, vp, i32, vp, vp, vp,
                                     vp, vp]
@@ -62,8 +62,8 @@ def bind(path: str) -> ctypes.CDLL:
     L.specext_prefill_attn.restype = ctypes.c_int
     L.specext_prefill_attn.argtypes = [ctypes.POINTER(AttnDesc)] + [vp] * 7
     L.specext_select_gather.restype = ctypes.c_int
-    L.specext_select_gather.argtypes = [vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, i32, i64, i64, i64,
-                                        vp, vp, vp, vp, vp, vp, vp]
+    L.specext_select_gather.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp, i32, i32, i32, i64, i64,
+                                        i64, vp, vp, vp, vp, vp, vp, vp]
     L.specext_read_status.restype = ctypes.c_int
     L.specext_read_status.argtypes = [vp, vp]
     L.specext_status_string.restype = ctypes.c_char_p
@@ -210,7 +210,8 @@ def specext_verify_attn_static_scratch(desc: AttnDesc, Q: torch.Tensor, K_prefix
 
 
 def specext_select_chunks(chunk_score: torch.Tensor, row: int, prefix_len: int, chunk_size: int, k: int,
-                          idx: torch.Tensor, n_selected: torch.Tensor, device_status: torch.Tensor) -> None:
+                          idx: torch.Tensor, n_selected: torch.Tensor, device_status: torch.Tensor,
+                          n_sink_chunks: int = 0, n_recent_chunks: int = 0) -> None:
     """Enqueues SelectChunks for one row of chunk_score [n_tree][n_chunks]."""
     if chunk_score.dtype != torch.float32 or chunk_score.dim() != 2 or not chunk_score.is_contiguous():
         raise ValueError("chunk_score must be a contiguous fp32 [n_tree][n_chunks] tensor")
@@ -220,7 +221,8 @@ def specext_select_chunks(chunk_score: torch.Tensor, row: int, prefix_len: int, 
     if idx.numel() < min(k, n_chunks):
         raise ValueError("idx is too small")
     rc = lib().specext_select_chunks(_ptr(chunk_score), n_tree, n_chunks, int(row), int(prefix_len),
-                                     int(chunk_size), int(k), _ptr(idx), _ptr(n_selected),
+                                     int(chunk_size), int(k), int(n_sink_chunks), int(n_recent_chunks),
+                                     _ptr(idx), _ptr(n_selected),
                                      _ptr(device_status), _stream())
     _check(rc, "specext_select_chunks")
 
@@ -248,7 +250,8 @@ def specext_gather_kv(draft_K: torch.Tensor, draft_V: torch.Tensor, prefix_len: 
 def specext_select_gather(chunk_score: torch.Tensor, row: int, prefix_len: int, chunk_size: int, k: int,
                           draft_K: torch.Tensor, draft_V: torch.Tensor, idx: torch.Tensor,
                           n_selected: torch.Tensor, K_out: torch.Tensor, V_out: torch.Tensor,
-                          n_tokens_out: torch.Tensor, device_status: torch.Tensor) -> None:
+                          n_tokens_out: torch.Tensor, device_status: torch.Tensor, n_sink_chunks: int = 0,
+                          n_recent_chunks: int = 0) -> None:
     """Enqueues SelectChunks + UpdateDraftCache as one call (one kernel launch for the usual sizes)."""
     if chunk_score.dtype != torch.float32 or chunk_score.dim() != 2 or not chunk_score.is_contiguous():
         raise ValueError("chunk_score must be a contiguous fp32 [n_tree][n_chunks] tensor")
@@ -267,7 +270,8 @@ def specext_select_gather(chunk_score: torch.Tensor, row: int, prefix_len: int, 
     if not (K_out.is_contiguous() and V_out.is_contiguous()) or K_out.numel() < need or V_out.numel() < need:
         raise ValueError("K_out/V_out must be contiguous and hold [layers][k*C][H][D]")
     rc = lib().specext_select_gather(_ptr(chunk_score), n_tree, n_chunks, int(row), int(prefix_len),
-                                     int(chunk_size), int(k), _ptr(draft_K), _ptr(draft_V), nl, H, D,
+                                     int(chunk_size), int(k), int(n_sink_chunks), int(n_recent_chunks),
+                                     _ptr(draft_K), _ptr(draft_V), nl, H, D,
                                      draft_K.stride(0), draft_K.stride(1), draft_K.stride(2), _ptr(idx),
                                      _ptr(n_selected), _ptr(K_out), _ptr(V_out), _ptr(n_tokens_out),
                                      _ptr(device_status), _stream())

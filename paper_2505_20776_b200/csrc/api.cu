@@ -5,8 +5,8 @@
 
 #include "common.cuh"
 
-cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
-                              int32_t* n_selected, cudaStream_t st);
+cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int n_sink, int n_recent,
+                              int32_t* idx, int32_t* n_selected, cudaStream_t st);
 cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int H, int D, int L, int C,
                               long long s_layer, long long s_l, long long s_h, const int32_t* idx,
                               const int32_t* n_selected, int max_selected, void* K_out, void* V_out,
@@ -16,7 +16,8 @@ cudaError_t spx_launch_prefill_tc2(const void* Q, const void* K, const void* V, 
                                    long long kv_sh, long long o_st, long long o_sh, int n_sm, int32_t* status,
                                    cudaStream_t st);
 bool spx_select_gather_fusable(int NC, int k);
-cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* dK, const void* dV, int n_layers,
+cudaError_t spx_launch_select_gather(const float* score_row, int k, int n_sink, int n_recent, const void* dK,
+                                     const void* dV, int n_layers,
                                      int H, int D, int L, int C, long long s_layer, long long s_l, long long s_h,
                                      int32_t* idx, int32_t* n_selected, void* K_out, void* V_out,
                                      int32_t* n_tokens_out, int32_t* status, cudaStream_t st);
@@ -313,11 +314,13 @@ int specext_verify_attn_static_scratch(const specext_attn_desc* desc, const void
 }
 
 int specext_select_chunks(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
-                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t* idx,
-                          int32_t* n_selected, int32_t* device_status, void* cuda_stream) {
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t n_sink_chunks,
+                          int32_t n_recent_chunks, int32_t* idx, int32_t* n_selected, int32_t* device_status,
+                          void* cuda_stream) {
   (void)device_status;
   if (!idx || !n_selected) return SPECEXT_ERR_INVALID_ARG;
-  if (n_tree < 1 || row < 0 || row >= n_tree || k < 1 || chunk_size < 1 || prefix_len < 0)
+  if (n_tree < 1 || row < 0 || row >= n_tree || k < 1 || chunk_size < 1 || prefix_len < 0 || n_sink_chunks < 0 ||
+      n_recent_chunks < 0)
     return SPECEXT_ERR_INVALID_ARG;
   const long long nc = ((long long)prefix_len + chunk_size - 1) / chunk_size;
   if (nc != n_chunks) return SPECEXT_ERR_INVALID_ARG;
@@ -328,8 +331,8 @@ int specext_select_chunks(const float* chunk_score, int32_t n_tree, int32_t n_ch
     e = cudaMemsetAsync(n_selected, 0, sizeof(int32_t), st);
   } else {
     if (!chunk_score) return SPECEXT_ERR_INVALID_ARG;
-    e = spx_launch_select(chunk_score + (long long)row * n_chunks, n_chunks, prefix_len, chunk_size, k, idx,
-                          n_selected, st);
+    e = spx_launch_select(chunk_score + (long long)row * n_chunks, n_chunks, prefix_len, chunk_size, k,
+                          n_sink_chunks, n_recent_chunks, idx, n_selected, st);
     g_launches.fetch_add(1);
   }
   if (e != cudaSuccess) {
@@ -361,18 +364,19 @@ int specext_gather_kv(const void* draft_K, const void* draft_V, int32_t n_layers
 }
 
 int specext_select_gather(const float* chunk_score, int32_t n_tree, int32_t n_chunks, int32_t row,
-                          int32_t prefix_len, int32_t chunk_size, int32_t k, const void* draft_K,
+                          int32_t prefix_len, int32_t chunk_size, int32_t k, int32_t n_sink_chunks,
+                          int32_t n_recent_chunks, const void* draft_K,
                           const void* draft_V, int32_t n_layers, int32_t n_kv_heads, int32_t head_dim,
                           int64_t stride_layer, int64_t stride_l, int64_t stride_h, int32_t* idx,
                           int32_t* n_selected, void* K_out, void* V_out, int32_t* n_tokens_out,
                           int32_t* device_status, void* cuda_stream) {
   const long long nc = chunk_size >= 1 && prefix_len >= 0 ? ((long long)prefix_len + chunk_size - 1) / chunk_size : -1;
   const bool fuse = nc == n_chunks && n_tree >= 1 && row >= 0 && row < n_tree && k >= 1 && chunk_score &&
-                    spx_select_gather_fusable(n_chunks, k);
+                    n_sink_chunks >= 0 && n_recent_chunks >= 0 && spx_select_gather_fusable(n_chunks, k);
   if (!fuse) {
     // sizes the single launch is not built for, and every invalid argument, take the two calls
-    const int rc = specext_select_chunks(chunk_score, n_tree, n_chunks, row, prefix_len, chunk_size, k, idx,
-                                         n_selected, device_status, cuda_stream);
+    const int rc = specext_select_chunks(chunk_score, n_tree, n_chunks, row, prefix_len, chunk_size, k,
+                                         n_sink_chunks, n_recent_chunks, idx, n_selected, device_status, cuda_stream);
     if (rc != SPECEXT_OK) return rc;
     return specext_gather_kv(draft_K, draft_V, n_layers, n_kv_heads, head_dim, prefix_len, chunk_size, stride_layer,
                              stride_l, stride_h, idx, n_selected, k, K_out, V_out, n_tokens_out, device_status,
@@ -383,7 +387,8 @@ int specext_select_gather(const float* chunk_score, int32_t n_tree, int32_t n_ch
                                    stride_layer, stride_l, stride_h, k, K_out, V_out, n_tokens_out);
   if (rc != SPECEXT_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const cudaError_t e = spx_launch_select_gather(chunk_score + (long long)row * n_chunks, k, draft_K, draft_V,
+  const cudaError_t e = spx_launch_select_gather(chunk_score + (long long)row * n_chunks, k, n_sink_chunks,
+                                                 n_recent_chunks, draft_K, draft_V,
                                                  n_layers, n_kv_heads, head_dim, prefix_len, chunk_size,
                                                  stride_layer, stride_l, stride_h, idx, n_selected, K_out, V_out,
                                                  n_tokens_out, device_status, st);

@@ -18,10 +18,18 @@ constexpr int kFusedThreads = 256;
 constexpr int kFusedMaxK = 1024;           // selected indices a fused block keeps in shared memory
 constexpr int kFusedMaxChunks = 8192;      // above this every block repeating the selection costs more than a launch
 
-__device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, int c, int NC, int L, int C) {
-  const int len = (c == NC - 1) ? (L - c * C) : C;
+// Shape of one selection: chunk count, prefix length, chunk size, and the forced chunks (the first n_sink
+// and the last n_recent chunks are kept whatever their score; 0 and 0 = the plain top-k).
+struct SelShape {
+  int NC, L, C, n_sink, n_recent;
+};
+
+__device__ __forceinline__ uint32_t chunk_key(const float* __restrict__ score, int c, const SelShape& sh) {
+  if (c < sh.n_sink || c >= sh.NC - sh.n_recent) return 0x7F800000u;     // +inf: above every finite key, ties by index
+  const int len = (c == sh.NC - 1) ? (sh.L - c * sh.C) : sh.C;
   float x = score[c] / (float)len;
   if (!(x > 0.f)) x = 0.f;                 // -0, negative or NaN rank lowest
+  if (x > 3.0e38f) x = 3.0e38f;            // a finite score never reaches the forced chunks' key
   return __float_as_uint(x);
 }
 
@@ -39,15 +47,16 @@ struct SelectSmem {
 // to idx_out (global or shared memory).  Every thread of the block must call it.  Two block barriers per
 // radix pass and two per batch of NT chunks in the emission.
 template <int NT>
-__device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __restrict__ score, int NC, int L,
-                                             int C, int keff, int32_t* idx_out) {
+__device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __restrict__ score, const SelShape& sh,
+                                             int keff, int32_t* idx_out) {
+  const int NC = sh.NC;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int NW = NT / 32;
   // one load and one division per chunk when the keys fit in shared memory
   const bool cached = NC <= kKeyCache;
   if (cached)
-    for (int c = tid; c < NC; c += NT) sm.keys[c] = chunk_key(score, c, NC, L, C);
-  auto key_of = [&](int c) -> uint32_t { return cached ? sm.keys[c] : chunk_key(score, c, NC, L, C); };
+    for (int c = tid; c < NC; c += NT) sm.keys[c] = chunk_key(score, c, sh);
+  auto key_of = [&](int c) -> uint32_t { return cached ? sm.keys[c] : chunk_key(score, c, sh); };
   for (int i = tid; i < 4 * 256; i += NT) (&sm.hist[0][0])[i] = 0;
   __syncthreads();
 
@@ -133,13 +142,13 @@ __device__ __forceinline__ void select_block(SelectSmem<NT>& sm, const float* __
 }
 
 template <int NT>
-__global__ void __launch_bounds__(NT) select_kernel(const float* __restrict__ score, int NC, int L, int C, int k,
+__global__ void __launch_bounds__(NT) select_kernel(const float* __restrict__ score, const SelShape sh, int k,
                                                     int32_t* __restrict__ idx, int32_t* __restrict__ n_selected) {
   __shared__ SelectSmem<NT> sm;
   sm100::pdl_launch_dependents();
   sm100::pdl_wait();                       // the scores are complete
-  const int keff = min(k, NC);
-  select_block<NT>(sm, score, NC, L, C, keff, idx);
+  const int keff = min(k, sh.NC);
+  select_block<NT>(sm, score, sh, keff, idx);
   if (threadIdx.x == 0) *n_selected = keff;
 }
 
@@ -156,7 +165,7 @@ struct GatherArgs {
   const float* score;
   int32_t* idx_out;
   int32_t* n_selected_out;
-  int k;
+  int k, n_sink, n_recent;
 };
 
 // Copies the tokens [o_lo, o_hi) of kept chunk number i (chunk index c) of one layer of K or V.
@@ -246,7 +255,8 @@ __global__ void __launch_bounds__(kFusedThreads) select_gather_kernel(const __gr
   sm100::pdl_wait();                                 // the scores are complete
   const int keff = min(g.k, g.NC);
   if (i >= keff) return;                             // uniform for the block
-  select_block<kFusedThreads>(sm, g.score, g.NC, g.L, g.C, keff, s_idx);
+  const SelShape sh = {g.NC, g.L, g.C, g.n_sink, g.n_recent};
+  select_block<kFusedThreads>(sm, g.score, sh, keff, s_idx);
   __syncthreads();
   if (blockIdx.x == 0 && layer == 0 && which == 0) {
     for (int j = threadIdx.x; j < keff; j += kFusedThreads) g.idx_out[j] = s_idx[j];
@@ -292,14 +302,15 @@ void fill_gather_args(GatherArgs& g, const void* dK, const void* dV, int n_layer
   g.sub = sub;
   g.s_layer = s_layer; g.s_l = s_l; g.s_h = s_h;
   g.idx = nullptr; g.n_selected = nullptr;
-  g.score = nullptr; g.idx_out = nullptr; g.n_selected_out = nullptr; g.k = 0;
+  g.score = nullptr; g.idx_out = nullptr; g.n_selected_out = nullptr; g.k = 0; g.n_sink = 0; g.n_recent = 0;
 }
 
 }  // namespace
 
-cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int32_t* idx,
-                              int32_t* n_selected, cudaStream_t st) {
-  void* args[] = {&score_row, &NC, &L, &C, &k, &idx, &n_selected};
+cudaError_t spx_launch_select(const float* score_row, int NC, int L, int C, int k, int n_sink, int n_recent,
+                              int32_t* idx, int32_t* n_selected, cudaStream_t st) {
+  SelShape sh = {NC, L, C, n_sink, n_recent};
+  void* args[] = {&score_row, &sh, &k, &idx, &n_selected};
   // few chunks: a small block, whose barriers are cheap; many: the widest one
   if (NC <= 2048)
     return launch_pdl(reinterpret_cast<const void*>(select_kernel<kFusedThreads>), dim3(1), dim3(kFusedThreads), args, st);
@@ -323,7 +334,8 @@ cudaError_t spx_launch_gather(const void* dK, const void* dV, int n_layers, int 
 // True when SelectChunks + UpdateDraftCache of this size run as one launch.
 bool spx_select_gather_fusable(int NC, int k) { return NC >= 1 && NC <= kFusedMaxChunks && k <= kFusedMaxK; }
 
-cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* dK, const void* dV, int n_layers,
+cudaError_t spx_launch_select_gather(const float* score_row, int k, int n_sink, int n_recent, const void* dK,
+                                     const void* dV, int n_layers,
                                      int H, int D, int L, int C, long long s_layer, long long s_l, long long s_h,
                                      int32_t* idx, int32_t* n_selected, void* K_out, void* V_out,
                                      int32_t* n_tokens_out, int32_t* status, cudaStream_t st) {
@@ -333,6 +345,8 @@ cudaError_t spx_launch_select_gather(const float* score_row, int k, const void* 
   g.idx_out = idx;
   g.n_selected_out = n_selected;
   g.k = k;
+  g.n_sink = n_sink;
+  g.n_recent = n_recent;
   void* args[] = {&g};
   const int keff = k < g.NC ? k : g.NC;
   return launch_pdl(reinterpret_cast<const void*>(select_gather_kernel), dim3(keff * g.sub, n_layers, 2),

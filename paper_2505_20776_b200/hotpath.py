@@ -76,19 +76,20 @@ class HotPath:
         api.specext_verify_attn(d, t["Q"], t["K_prefix"], t["V_prefix"], t["K_tree"], t["V_tree"], parent,
                                 self.O, self.lse, cs, self._ws, self.status)
 
-    def select_chunks(self, row: int, prefix_len: int) -> None:
+    def select_chunks(self, row: int, prefix_len: int, n_sink_chunks: int = 0, n_recent_chunks: int = 0) -> None:
         api.specext_select_chunks(self.chunk_score(prefix_len), row, prefix_len, self.C, self.k, self.idx,
-                                  self.n_selected, self.status)
+                                  self.n_selected, self.status, n_sink_chunks, n_recent_chunks)
 
     def gather_kv(self, draft_K: torch.Tensor, draft_V: torch.Tensor, prefix_len: int) -> None:
         api.specext_gather_kv(draft_K, draft_V, prefix_len, self.C, self.idx, self.n_selected, self.k,
                               self.K_compact, self.V_compact, self.n_tokens, self.status)
 
-    def select_gather(self, row: int, prefix_len: int, draft_K: torch.Tensor, draft_V: torch.Tensor) -> None:
+    def select_gather(self, row: int, prefix_len: int, draft_K: torch.Tensor, draft_V: torch.Tensor,
+                      n_sink_chunks: int = 0, n_recent_chunks: int = 0) -> None:
         """SelectChunks + UpdateDraftCache as one library call."""
         api.specext_select_gather(self.chunk_score(prefix_len), row, prefix_len, self.C, self.k, draft_K, draft_V,
                                   self.idx, self.n_selected, self.K_compact, self.V_compact, self.n_tokens,
-                                  self.status)
+                                  self.status, n_sink_chunks, n_recent_chunks)
 
     def read_status(self) -> int:
         return api.specext_read_status(self.status)

@@ -78,7 +78,7 @@ def test_host_side_rejection_needs_no_gpu(lib):
     d = _desc()
     rc = lib.specext_verify_attn(ctypes.byref(d), *([None] * 9), None, 0, None, None)
     assert rc == 1                                            # null pointers
-    assert lib.specext_select_chunks(None, 4, 8, 0, 256, 32, 4, None, None, None, None) == 1
-    assert lib.specext_select_gather(None, 4, 8, 0, 256, 32, 4, *([None] * 2), 1, 8, 128, 0, 1024, 128, *([None] * 7)) == 1
+    assert lib.specext_select_chunks(None, 4, 8, 0, 256, 32, 4, 0, 0, None, None, None, None) == 1
+    assert lib.specext_select_gather(None, 4, 8, 0, 256, 32, 4, 0, 0, *([None] * 2), 1, 8, 128, 0, 1024, 128, *([None] * 7)) == 1
     assert lib.specext_status_string(4).decode().startswith("parent")
     assert lib.specext_launch_count() >= 0

@@ -321,6 +321,43 @@ def test_select_bit_exact_on_given_scores(cuda_device):
         check_select_bit_exact(hp, np.full(NC, 0.25, dtype=np.float32), L, C, k)
 
 
+def test_forced_sink_and_recent_chunks(cuda_device):
+    """The extension of SelectChunks (earliest / latest chunks kept whatever their score), on given fp32 score
+    rows: indices bit-exact with the oracle through both the two-call and the one-call route, gathered cache
+    bit-exact with the oracle's gather."""
+    dev = cuda_device
+    rng = np.random.default_rng(17)
+    for NC, C, tail in [(128, 32, 0), (333, 8, 5), (9000, 1, 0)]:
+        L = NC * C - tail
+        w = _small(4, 2, 128, L, 2, C, k=1)
+        dK, dV = synth.make_draft_kv(w)
+        dKd, dVd = dK.to(dev), dV.to(dev)
+        for n_sink, n_recent, k in [(1, 0, 8), (0, 2, 8), (2, 2, 8), (4, 4, 6), (3, 1, 3), (0, 0, 8)]:
+            hp = GuardedHotPath(4, 2, 128, 2, C, k, L, device=dev)
+            score = rng.random(NC).astype(np.float32)
+            cs = hp.chunk_score(L)
+            cs.zero_()
+            cs[1] = torch.from_numpy(score).to(dev)
+            want = orc.select_chunks(score, L, C, k, key_dtype=np.float32, n_sink=n_sink, n_recent=n_recent)
+            Kr, Vr, ntok = orc.gather_kv(dK.view(torch.int16).numpy(), dV.view(torch.int16).numpy(), want, L, C)
+            for one_call in (False, True):
+                hp.idx.fill_(-1)
+                hp.K_compact.zero_()
+                if one_call:
+                    hp.select_gather(1, L, dKd, dVd, n_sink, n_recent)
+                else:
+                    hp.select_chunks(1, L, n_sink, n_recent)
+                    hp.gather_kv(dKd, dVd, L)
+                assert hp.read_status() == 0
+                hp.check()
+                assert int(hp.n_selected.item()) == len(want) and int(hp.n_tokens.item()) == ntok
+                np.testing.assert_array_equal(hp.idx[: len(want)].cpu().numpy(), want)
+                np.testing.assert_array_equal(bf16_bits(hp.K_compact)[:, :ntok], Kr)
+                np.testing.assert_array_equal(bf16_bits(hp.V_compact)[:, :ntok], Vr)
+            forced = set(range(n_sink)) | set(range(NC - n_recent, NC))
+            assert len(forced) > k or forced <= set(want.tolist())
+
+
 def test_bad_tree_sets_status(cuda_device):
     w = _small(4, 1, 64, 64, 4, 32)
     dev = cuda_device
