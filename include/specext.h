@@ -51,7 +51,7 @@ typedef struct {
   int32_t n_kv_heads;      /* Hkv; Hq % Hkv == 0 and G = Hq/Hkv a power of two <= 64          */
   int32_t head_dim;        /* D: 64 or 128                                                    */
   int32_t prefix_len;      /* L >= 0: number of valid tokens in the prefix KV cache           */
-  int32_t n_tree;          /* T: draft-tree nodes, 1..64                                      */
+  int32_t n_tree;          /* T: draft-tree nodes, 1..128                                     */
   int32_t chunk_size;      /* C: tokens per retrieval chunk, a power of two in 1..128         */
   float softmax_scale;     /* multiplies q.k before the softmax; 0 selects 1/sqrt(D)          */
   int32_t want_chunk_score;/* non-zero: also produce chunk_score (the last layer only)        */

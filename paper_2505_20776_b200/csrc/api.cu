@@ -70,7 +70,7 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   if (!d) return SPECEXT_ERR_INVALID_ARG;
   if (d->n_q_heads < 1 || d->n_kv_heads < 1 || d->n_q_heads % d->n_kv_heads != 0) return SPECEXT_ERR_INVALID_ARG;
   if (d->prefix_len < 0 || d->prefix_len > (1 << 24)) return SPECEXT_ERR_INVALID_ARG;
-  if (d->n_tree < 1 || d->n_tree > 64) return SPECEXT_ERR_UNSUPPORTED;
+  if (d->n_tree < 1 || d->n_tree > kSpxMaxTree) return SPECEXT_ERR_UNSUPPORTED;
   if (d->head_dim != 64 && d->head_dim != 128) return SPECEXT_ERR_UNSUPPORTED;
   if (!is_pow2(d->chunk_size) || d->chunk_size > 128) return SPECEXT_ERR_UNSUPPORTED;
   const int G = d->n_q_heads / d->n_kv_heads;
@@ -86,7 +86,9 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   p.Hq = d->n_q_heads; p.Hkv = d->n_kv_heads; p.G = G; p.D = d->head_dim;
   p.L = d->prefix_len; p.T = d->n_tree; p.C = d->chunk_size;
   p.rows = G * p.T;
-  p.RB = p.rows > 128 ? 256 : 128;
+  // (a tree of more than 64 nodes with head_dim 128 always takes 256-row blocks: the one-CTA kernel keeps
+  // one mask word per node there)
+  p.RB = (p.rows > 128 || (p.D == 128 && p.T > 64)) ? 256 : 128;
   p.n_rblk = (p.rows + p.RB - 1) / p.RB;
   p.NP = p.Hkv * p.n_rblk;
   p.TPH = (p.L + SPX_TILE_KEYS - 1) / SPX_TILE_KEYS;
@@ -98,6 +100,7 @@ int build_plan(const specext_attn_desc* d, AttnPlan* out) {
   const int want = tuning_kernel();
   const bool pair_ok = p.D == 128 && p.RB == 256;       // what the paired-CTA kernel is built for
   p.kernel = want == 1 ? 1 : ((want == 0 || want == 3) && pair_ok ? 3 : 2);   // want != 0 only in the test library
+  if (p.kernel == 2 && p.D == 128 && p.T > 64) return SPECEXT_ERR_UNSUPPORTED;  // (only reachable by a test override)
   if (p.kernel == 3) {
     // one worker = a cluster of two CTAs; every problem gets the same number of workers when possible
     const int n_workers = sm_count() / 2 > 0 ? sm_count() / 2 : 1;

@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(const __grid_constant__ 
       }
     }
     float m = -INFINITY, l = 0.f;
-    const unsigned long long my_anc = anc[t];
+    const unsigned long long my_anc_lo = anc[2 * t], my_anc_hi = anc[2 * t + 1];
 
     for (int tile = tile_lo; tile < tile_hi; ++tile) {
       const bool is_tree = tile == p.TPH;
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(const __grid_constant__ 
         acc += __shfl_xor_sync(0xffffffffu, acc, 1);
         acc += __shfl_xor_sync(0xffffffffu, acc, 2);
         float s = acc * p.scale2;
-        const bool vis = (j < nkeys) && (!is_tree || ((my_anc >> j) & 1ull));
+        const bool vis = (j < nkeys) && (!is_tree || (((j < 64 ? my_anc_lo >> j : my_anc_hi >> (j - 64)) & 1ull) != 0));
         s = vis ? s : -INFINITY;
         tmax = fmaxf(tmax, s);
         if (quarter == 0) S[row_local * kSStride + j] = s;
@@ -154,7 +154,7 @@ cudaError_t spx_launch_attn_simt(const AttnArgs& a, cudaStream_t st, int* n_laun
   const AttnPlan& p = a.plan;
   const dim3 grid(p.n_cta, p.RB / kRowsPerCta);
   const size_t smem = 2ull * SPX_TILE_KEYS * p.D * sizeof(__nv_bfloat16) +
-                      kRowsPerCta * kSStride * sizeof(float) + 64 * sizeof(unsigned long long);
+                      kRowsPerCta * kSStride * sizeof(float) + 2 * kSpxMaxTree * sizeof(unsigned long long);
   cudaError_t e;
   if (p.D == 128) {
     e = cudaFuncSetAttribute(attn_simt_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

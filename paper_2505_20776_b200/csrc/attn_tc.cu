@@ -49,19 +49,27 @@ struct Cfg {
   static constexpr int kQBytes = 2 * DS * kSubTileBytes;      // two row tiles
   static constexpr int kStages = D == 128 ? 5 : 8;
   static constexpr int kBarOffset = kQBytes + kStages * kStageBytes;
-  static constexpr int kSmemBytes = kBarOffset + 1024 + 1024; // + control block + alignment slack
+  // Trees of more than 64 nodes need two mask words per node.  With head_dim 128 the rings leave only 1 KB
+  // for the control block, and such a tree with at most 128 stacked rows (one query head per KV head) is sent
+  // to the paired kernel by the plan; with head_dim 64 there is room for the full 128 nodes.
+  static constexpr int kTreeMax = D == 128 ? 64 : kSpxMaxTree;
+  static constexpr int kCtrlBytes = D == 128 ? 1024 : 3072;
+  static constexpr int kSmemBytes = kBarOffset + kCtrlBytes + 1024; // + control block + alignment slack
 };
 
-struct Ctrl {
+template <int D>
+struct CtrlT {
   uint64_t q_full, q_free, drain;
   uint64_t v_rag;                 // a V tile whose tail rows must be cleared has landed (device-side length)
   uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
   uint64_t kv_full[8], kv_empty[8];
-  unsigned long long anc[64];
-  int parent[64];
+  unsigned long long anc[Cfg<D>::kTreeMax][Cfg<D>::kTreeMax / 64];
+  int parent[Cfg<D>::kTreeMax];
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(CtrlT<128>) <= Cfg<128>::kCtrlBytes && sizeof(CtrlT<64>) <= Cfg<64>::kCtrlBytes,
+              "control block too large");
 
 // DEVLEN: the prefix length is read from device memory (a.L_dev) and may be shorter than the planned
 // capacity p.L; the instantiation without it carries none of that code.
@@ -78,6 +86,8 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
                                                          ~static_cast<uintptr_t>(1023));
   unsigned char* Qs = base;
   unsigned char* ring = base + C::kQBytes;
+  using Ctrl = CtrlT<D>;
+  constexpr int kTreeMax = C::kTreeMax;
   Ctrl* ctl = reinterpret_cast<Ctrl*>(base + C::kBarOffset);
   volatile int* abort_flag = &ctl->abort_flag;
 
@@ -199,23 +209,17 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
       tmem_alloc(&ctl->tmem_base, 512);
       tmem_relinquish();
     } else if (warp > kMmaWarp) {
-      const int t = tid - (kMmaWarp + 1) * 32;                  // 0..63
-      ctl->parent[t] = t < p.T ? a.parent[t] : -1;
+      const int t64 = tid - (kMmaWarp + 1) * 32;                // 0..63
+      for (int t = t64; t < kTreeMax; t += 64) ctl->parent[t] = t < p.T ? a.parent[t] : -1;
       named_bar_sync(2, 64);
-      unsigned long long m = 0;
-      if (t < p.T) {
-        int u = t;
-        for (int step = 0; step <= p.T && u >= 0; ++step) {
-          m |= 1ull << u;
-          const int pu = ctl->parent[u];
-          if (pu < -1 || pu >= u) {
-            if (cta == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
-            break;
-          }
-          u = pu;
-        }
+      bool bad = false;
+      for (int t = t64; t < kTreeMax; t += 64) {
+        SpxMask128 m = {0ull, 0ull};
+        if (t < p.T) m = spx_walk_up(ctl->parent, p.T, t, bad);
+        ctl->anc[t][0] = m.lo;
+        if (kTreeMax > 64) ctl->anc[t][kTreeMax / 64 - 1] = m.hi;
       }
-      ctl->anc[t] = m;
+      if (bad && cta == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
     }
     tc_fence_before();
     named_bar_sync(1, kThreads - 32);
@@ -350,7 +354,7 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             u += n_units;
             continue;
           }
-          const unsigned long long tree_mask = valid ? ctl->anc[r / p.G] : 1ull;
+          const int t_node = valid ? r / p.G : 0;
           float m_used = -INFINITY, l = 0.f;
 
           for (int jt = 0; jt < n_seg; ++jt, ++it) {
@@ -371,9 +375,9 @@ attn_tc_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ TcMap
             tmem_wait_ld();
             if (need_mask) {
               unsigned long long vis_lo, vis_hi;
-              if (is_tree) {
-                vis_lo = tree_mask;
-                vis_hi = 0ull;
+              if (is_tree) {               // this node and its ancestors (a padding row sees key 0)
+                vis_lo = valid ? ctl->anc[t_node][0] : 1ull;
+                vis_hi = (kTreeMax > 64 && valid) ? ctl->anc[t_node][kTreeMax / 64 - 1] : 0ull;
               } else {
                 vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
                 vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);

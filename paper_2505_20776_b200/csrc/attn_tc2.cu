@@ -50,7 +50,7 @@ constexpr int D = 128;
 constexpr int kStageBytes = 16384;             // half of a K tile (64 keys x 128) or of a V tile (128 keys x 64)
 constexpr int kStages = 6;                     // per ring; one ring for K halves, one for V halves
 constexpr int kCtrlOffset = 2 * kStages * kStageBytes;
-constexpr int kSmemBytes = kCtrlOffset + 3072 + 1024;
+constexpr int kSmemBytes = kCtrlOffset + 4096 + 1024;
 constexpr float kRescaleThreshold = 8.0f;      // log2 units
 constexpr uint32_t kColO = 0, kColS = 128, kColQ = 384, kColP = 448;
 
@@ -71,14 +71,14 @@ struct Ctrl {
   uint64_t q_land;              // this CTA: the first segment's Q rows have landed in the scratch (TMA)
   uint64_t v_rag;               // this CTA: a V half whose tail rows must be cleared has landed (device-side length)
   uint64_t epi[2];              // this CTA: 8 arrivals, the two meeting points of a segment's epilogue
-  unsigned long long anc[64];
-  int parent[64];
+  unsigned long long anc[kSpxMaxTree][2];
+  int parent[kSpxMaxTree];
   float m_row[128];             // reference maximum of each row after the latest tile
   float l_x[128];               // epilogue: warpgroup 1 hands its row sums to warpgroup 0
   uint32_t tmem_base;
   int abort_flag;
 };
-static_assert(sizeof(Ctrl) <= 3072, "control block too large");
+static_assert(sizeof(Ctrl) <= 4096, "control block too large");
 
 // SCORE: 0 no chunk sums; otherwise the class of the chunk size, so that each variant carries only the
 // code it runs (the loop of the exponentials is instruction-cache sensitive): 1 chunks of 32 keys,
@@ -359,27 +359,19 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
     if (warp == kTreeWarp) {
       // registers first: the softmax warpgroups cannot grow until every warp of this warpgroup has shrunk
       setmaxnreg_dec<kRegsOther>();
-      ctl->parent[lane] = lane < p.T ? a.parent[lane] : -1;
-      ctl->parent[lane + 32] = lane + 32 < p.T ? a.parent[lane + 32] : -1;
-      __syncwarp();
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int t = lane + 32 * half;
-        unsigned long long m = 0;
-        if (t < p.T) {
-          int u = t;
-          for (int step = 0; step <= p.T && u >= 0; ++step) {
-            m |= 1ull << u;
-            const int pu = ctl->parent[u];
-            if (pu < -1 || pu >= u) {
-              if (blockIdx.x == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
-              break;
-            }
-            u = pu;
-          }
-        }
-        ctl->anc[t] = m;
+      for (int q = 0; q < kSpxMaxTree / 32; ++q) ctl->parent[lane + 32 * q] = lane + 32 * q < p.T ? a.parent[lane + 32 * q] : -1;
+      __syncwarp();
+      bool bad = false;
+#pragma unroll 1
+      for (int q = 0; q < kSpxMaxTree / 32; ++q) {
+        const int t = lane + 32 * q;
+        SpxMask128 m = {0ull, 0ull};
+        if (t < p.T) m = spx_walk_up(ctl->parent, p.T, t, bad);
+        ctl->anc[t][0] = m.lo;
+        ctl->anc[t][1] = m.hi;
       }
+      if (bad && blockIdx.x == 0) spx_raise(a.status, SPECEXT_ERR_BAD_TREE);
       cluster_wait();                      // this CTA's barriers exist
       warp_arrive(&ctl->anc_ready, lane);
     }
@@ -564,7 +556,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           if (!ok) break;
           anc_seen = true;
         }
-        const unsigned long long tree_mask = valid ? ctl->anc[t_node] : 1ull;
 
         float m_loc = -INFINITY, l = 0.f;        // l is relative to m_loc
         for (int j = wg; j < n && ok; j += 2) {
@@ -585,9 +576,9 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           warp_arrive_cluster(s_free_l, lane);          // the S buffer may take the next tile
           if (need_mask) {
             unsigned long long vis_lo, vis_hi;
-            if (is_tree) {
-              vis_lo = tree_mask;
-              vis_hi = 0ull;
+            if (is_tree) {                 // this node and its ancestors (a padding row sees key 0)
+              vis_lo = valid ? ctl->anc[t_node][0] : 1ull;
+              vis_hi = valid ? ctl->anc[t_node][1] : 0ull;
             } else {
               vis_lo = nkeys >= 64 ? ~0ull : ((1ull << nkeys) - 1ull);
               vis_hi = nkeys <= 64 ? 0ull : ((1ull << (nkeys - 64)) - 1ull);

@@ -39,27 +39,38 @@ __device__ __forceinline__ int spx_prefix_len(const AttnArgs& a) {
   return v < 0 ? 0 : (v > a.plan.L ? a.plan.L : v);
 }
 
-// Ancestor-or-self bit masks of the draft tree: bit u of anc[t] is set iff u == t or u is a
-// proper ancestor of t.  Each of the first T threads walks up from its own node; a parent outside
-// [-1, t-1] raises BAD_TREE and ends the walk, so the loop is bounded by T steps.
+// Ancestor-or-self bit masks of the draft tree (up to kSpxMaxTree nodes, two 64-bit words per node): bit
+// u is set iff u == t or u is a proper ancestor of t.  The walk up from node t is bounded by T steps; a
+// parent outside [-1, u-1] ends it and is reported through `bad` (BAD_TREE).
+constexpr int kSpxMaxTree = 128;
+struct SpxMask128 {
+  unsigned long long lo, hi;
+};
+__device__ __forceinline__ SpxMask128 spx_walk_up(const int* parent, int T, int t, bool& bad) {
+  SpxMask128 m = {0ull, 0ull};
+  int u = t;
+  for (int step = 0; step <= T && u >= 0; ++step) {
+    if (u < 64) m.lo |= 1ull << u; else m.hi |= 1ull << (u - 64);
+    const int pu = parent[u];
+    if (pu < -1 || pu >= u) {
+      bad = true;
+      break;
+    }
+    u = pu;
+  }
+  return m;
+}
+// The masks of all nodes into shared memory (anc_smem[2*t], anc_smem[2*t+1]) by the first 128 threads.
 __device__ __forceinline__ void spx_build_ancestors(const int32_t* __restrict__ parent, int T,
                                                     unsigned long long* anc_smem, int32_t* status) {
   const int t = threadIdx.x;
-  if (t < 64) {
-    unsigned long long m = 0;
-    if (t < T) {
-      int u = t;
-      for (int step = 0; step <= T && u >= 0; ++step) {
-        m |= 1ull << u;
-        const int p = parent[u];
-        if (p < -1 || p >= u) {
-          spx_raise(status, SPECEXT_ERR_BAD_TREE);
-          break;
-        }
-        u = p;
-      }
-    }
-    anc_smem[t] = m;
+  if (t < kSpxMaxTree) {
+    SpxMask128 m = {0ull, 0ull};
+    bool bad = false;
+    if (t < T) m = spx_walk_up(parent, T, t, bad);
+    if (bad) spx_raise(status, SPECEXT_ERR_BAD_TREE);
+    anc_smem[2 * t] = m.lo;
+    anc_smem[2 * t + 1] = m.hi;
   }
 }
 

@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(64 * kScoreSlices) score_kernel(const __grid_c
   __shared__ float part[kScoreSlices][64][VW];
   sm100::pdl_launch_dependents();
   sm100::pdl_wait();                               // lse and the chunk sums are complete
-  const int t = threadIdx.x, slice = threadIdx.y;
+  const int t = blockIdx.z * 64 + threadIdx.x, slice = threadIdx.y;       // 64 tree nodes per block
   const int tile = blockIdx.x;
   const int c0 = blockIdx.y * VW;                  // first chunk of the group inside the tile
   float acc[VW];
@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(64 * kScoreSlices) score_kernel(const __grid_c
     }
   }
 #pragma unroll
-  for (int k = 0; k < VW; ++k) part[slice][t][k] = acc[k];
+  for (int k = 0; k < VW; ++k) part[slice][threadIdx.x][k] = acc[k];
   __syncthreads();
   if (slice == 0 && t < p.T) {
     const float inv = 1.f / (float)p.Hq;
@@ -165,7 +165,7 @@ __global__ void __launch_bounds__(64 * kScoreSlices) score_kernel(const __grid_c
     for (int k = 0; k < VW; ++k) {
       float sum = 0.f;
 #pragma unroll
-      for (int q = 0; q < kScoreSlices; ++q) sum += part[q][t][k];
+      for (int q = 0; q < kScoreSlices; ++q) sum += part[q][threadIdx.x][k];
       const int c = tile * p.CPT + c0 + k;
       if (c < p.NC) a.chunk_score[(long long)t * p.NC + c] = sum * inv;
     }
@@ -215,11 +215,11 @@ cudaError_t spx_launch_merge(const AttnArgs& a, cudaStream_t st, int* n_launches
   if (e != cudaSuccess) return e;
   if (p.want_score && p.NC > 0) {
     if (p.CPT >= 4) {
-      e = launch_score<4>(a, dim3(p.TPH, p.CPT / 4), st);
+      e = launch_score<4>(a, dim3(p.TPH, p.CPT / 4, (p.T + 63) / 64), st);
     } else if (p.CPT == 2) {
-      e = launch_score<2>(a, dim3(p.TPH, 1), st);
+      e = launch_score<2>(a, dim3(p.TPH, 1, (p.T + 63) / 64), st);
     } else {
-      e = launch_score<1>(a, dim3(p.TPH, 1), st);
+      e = launch_score<1>(a, dim3(p.TPH, 1, (p.T + 63) / 64), st);
     }
     *n_launches += 1;
   }

@@ -64,7 +64,7 @@ def test_workspace_size_and_descriptor_checks(lib):
     # the per-chunk sums for [Hq*T rows padded to 256 per KV head][NC] plus one reference maximum per
     # (row, 128-key tile) make up the difference
     assert full - without == 4 * (8 * 128 * 256 * 4 + 8 * 128 * 256)
-    for bad in (dict(head_dim=96), dict(n_tree=0), dict(n_tree=65), dict(chunk_size=3), dict(chunk_size=256),
+    for bad in (dict(head_dim=96), dict(n_tree=0), dict(n_tree=129), dict(chunk_size=3), dict(chunk_size=256),
                 dict(n_kv_heads=5), dict(prefix_len=-4), dict(q_stride_h=100), dict(kv_stride_l=12),
                 dict(softmax_scale=float("nan"))):
         assert api.specext_verify_attn_workspace(_desc(**bad)) == 0

@@ -51,6 +51,7 @@ SHAPES = [
     (32, 8, 128, 1, "chain", 2048),            # EAGLE-class single layer (the target's layer shape), decode
     (32, 8, 128, 12, "uniform", 2048),         # EAGLE-class, small tree: 48 stacked rows -> one-CTA kernel
     (32, 8, 128, 60, "levels", 2048),          # EAGLE-class, a full 60-node tree: 240 rows -> paired kernel
+    (32, 8, 128, 100, "uniform", 1024),        # a tree of more than 64 nodes: two row blocks
 ]
 
 

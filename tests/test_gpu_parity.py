@@ -252,6 +252,24 @@ def test_edge_shapes(cuda_device, Hq, Hkv, D, L, T, C):
         assert hp.read_status() == 0 and int(hp.n_selected.item()) == 0
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,L,T,C,tree", [
+    (32, 8, 128, 1000, 100, 32, "uniform"),   # 400 stacked rows: two row blocks on the paired kernel
+    (32, 8, 128, 700, 128, 32, "levels"),     # the largest tree
+    (4, 4, 128, 300, 128, 32, "chain"),       # one query head per KV head, head_dim 128: 256-row blocks, a 128-deep chain
+    (4, 4, 64, 300, 128, 16, "chain"),        # head_dim 64: the one-CTA kernel with two mask words per node
+    (8, 2, 64, 200, 65, 32, "uniform"),
+    (8, 2, 128, 0, 90, 32, "chain"),          # tree only: node i sees exactly nodes 0..i, across both mask words
+])
+def test_trees_of_more_than_64_nodes(cuda_device, Hq, Hkv, D, L, T, C, tree):
+    w = _small(Hq, Hkv, D, L, T, C, tree=tree, seed=300 + T)
+    hp = make_hp(w, cuda_device, max_prefix=max(L, 1))
+    t = synth.make_layer(w)
+    parent = synth.make_tree(w)
+    _, _, cs = check_attn(hp, t, parent, L, C, tag=f"tree{T}-D{D}")
+    if L > 0:
+        check_retrieval(hp, cs, [0, T // 2, T - 1], L, C, w.top_k, synth.make_draft_kv(w))
+
+
 def test_single_key_returns_value_exactly(cuda_device):
     w = _small(4, 1, 64, 0, 1, 32)
     hp = make_hp(w, cuda_device, max_prefix=1)
@@ -383,7 +401,7 @@ def test_host_validation(cuda_device):
         api.specext_verify_attn(desc, t["Q"], t["K_prefix"], t["V_prefix"], t["K_tree"], t["V_tree"], par, hp.O,
                                 hp.lse, None, workspace, hp.status)
     call(d)
-    for field, value, code in [("head_dim", 96, 2), ("n_tree", 65, 2), ("chunk_size", 48, 2),
+    for field, value, code in [("head_dim", 96, 2), ("n_tree", 129, 2), ("chunk_size", 48, 2),
                                ("n_kv_heads", 3, 1), ("kv_stride_l", 60, 1), ("prefix_len", -1, 1)]:
         bad = api.AttnDesc.from_buffer_copy(d)
         setattr(bad, field, value)
