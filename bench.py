@@ -236,8 +236,9 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="all", choices=["all", "c1", "c2", "c3", "c4"],
-                    help="which configurations are timed besides the c2 headline (c2 = headline only)")
+    ap.add_argument("--workload", default="all", choices=["all", "c1", "c2", "c3", "c4", "long"],
+                    help="which configurations are timed besides the c2 headline (c2 = headline only; long = the c3 "
+                         "shape at 64K and 128K keys, beyond the paper's configurations)")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -421,7 +422,7 @@ def main():
         # ---- the other configurations ------------------------------------------------------
         others = {}
         which = [] if args.workload == "c2" or args.layers > 0 else (
-            ["c1", "c3", "c4"] if args.workload == "all" else [args.workload])
+            ["c1", "c3", "c4"] if args.workload == "all" else [] if args.workload == "long" else [args.workload])
         for name in which:
             ww = synth.WORKLOADS[name]
             par_np = synth.make_tree(ww)
@@ -458,6 +459,28 @@ def main():
             assert hpo.read_status() == 0
             del bufs, hpo, ddK, ddV
             torch.cuda.empty_cache()
+
+        # ---- longer prefixes than the paper's configurations (same layer shape as c3) --------
+        if args.layers == 0 and args.workload in ("all", "long"):
+            ww = synth.WORKLOADS["c3"]
+            par_np = synth.make_tree(ww)
+            par = torch.from_numpy(par_np).to(dev)
+            for Lx in (65536, 131072):
+                bufs = [synth.make_layer(ww, layer=i, device=dev, capacity=Lx) for i in range(2)]   # 2 x 268 / 537 MB
+                hpo = HotPath(ww.n_q_heads, ww.n_kv_heads, ww.head_dim, ww.n_tree, ww.chunk_size, ww.top_k, Lx,
+                              device=dev)
+
+                def calls():
+                    for b in bufs:
+                        hpo.verify_attn(b, par, Lx, False)
+
+                call_us = part_us(calls, len(bufs))
+                nbytes, flops = layer_work(ww, par_np.tolist(), False, Lx)
+                others[f"long@{Lx}"] = {"prefix_len": Lx, "kv_copies_rotated": len(bufs), "attn_call_us": call_us,
+                                        "algorithmic_bytes": nbytes, "algorithmic_flops": flops}
+                assert hpo.read_status() == 0
+                del bufs, hpo
+                torch.cuda.empty_cache()
 
         # ---- end to end: host buffers, copies inside the timed region ----------------------
         e2e = None
