@@ -624,15 +624,16 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
             m_loc = m_new;
           }
           // Completion of the PV of tile j-1 (the other warpgroup's) is needed before O may be
-          // rescaled and before the P buffer may be overwritten.  The PV of this warpgroup's own
-          // previous tile (j-2) is waited for first: once it is complete so is every earlier one,
-          // which keeps the parity test on the other barrier unambiguous.
+          // rescaled and before the P buffer may be overwritten; the PVs complete in order, so every
+          // earlier one is complete then too.  One parity test on the other warpgroup's barrier is
+          // enough: its previous completion (tile j-3) was waited for at this warpgroup's previous tile,
+          // or lies in a segment whose end every thread has seen, and its next one (tile j+1) needs this
+          // tile's P, so the barrier is either one completion short of the one asked for or at it.
           const uint32_t n_prev_other = n_oth + ((j + 1) >> 1);      // tiles given to the other warpgroup before j
           bool pv_seen = false;
           auto wait_prev_pv = [&]() -> bool {
             if (pv_seen) return true;
             pv_seen = true;
-            if (n_mine > 0 && !wait_c(&ctl->pv_done[wg], (n_mine - 1) & 1, abort_flag)) return false;
             if (n_prev_other > 0 && !wait_c(&ctl->pv_done[wg ^ 1], (n_prev_other - 1) & 1, abort_flag)) return false;
             tc_fence_after();
             return true;

@@ -363,7 +363,8 @@ prefill_tc2_kernel(const __grid_constant__ PrefillArgs a, const __grid_constant_
           auto wait_prev_pv = [&]() -> bool {
             if (pv_seen) return true;
             pv_seen = true;
-            if (n_mine > 0 && !wait_c(&ctl->pv_done[wg], (n_mine - 1) & 1, abort_flag)) return false;
+            // (one parity test suffices: the other warpgroup's barrier is either one completion short of the
+            // one asked for or at it, and the PVs complete in order)
             if (n_prev_other > 0 && !wait_c(&ctl->pv_done[wg ^ 1], (n_prev_other - 1) & 1, abort_flag)) return false;
             tc_fence_after();
             return true;
