@@ -571,6 +571,15 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           tmem_ld32(s_addr + 32, s1);
           tmem_ld32(s_addr + 64, s2);
           tmem_ld32(s_addr + 96, s3);
+          // The row's reference maximum after the previous tile (handled by the other warpgroup) is fetched
+          // while the scores are on their way from tensor memory: it was published long before, as a rule.
+          float m_cur = -INFINITY;
+          if (j > 0) {
+            ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
+            if (!ok) break;
+            ++n_other;
+            m_cur = ctl->m_row[row_t];
+          }
           tmem_wait_ld();
           tc_fence_before();
           warp_arrive_cluster(s_free_l, lane);          // the S buffer may take the next tile
@@ -603,14 +612,6 @@ attn_tc2_kernel(const __grid_constant__ AttnArgs a, const __grid_constant__ Tc2M
           }
           const float m_tile = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * scale2;
 
-          // the row's reference maximum after the previous tile (handled by the other warpgroup)
-          float m_cur = -INFINITY;
-          if (j > 0) {
-            ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
-            if (!ok) break;
-            ++n_other;
-            m_cur = ctl->m_row[row_t];
-          }
           float m_new = m_cur;
           bool rescale = false;
           if (m_tile > m_cur + kRescaleThreshold || m_cur == -INFINITY) {

@@ -310,6 +310,14 @@ prefill_tc2_kernel(const __grid_constant__ PrefillArgs a, const __grid_constant_
           tmem_ld32(s_addr + 32, s1);
           tmem_ld32(s_addr + 64, s2);
           tmem_ld32(s_addr + 96, s3);
+          // the row's reference maximum after the previous tile is fetched while the scores are on their way
+          float m_cur = -INFINITY;
+          if (j > 0) {
+            ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
+            if (!ok) break;
+            ++n_other;
+            m_cur = ctl->m_row[row_t];
+          }
           tmem_wait_ld();
           tc_fence_before();
           warp_arrive_cluster(s_free_l, lane);
@@ -339,13 +347,6 @@ prefill_tc2_kernel(const __grid_constant__ PrefillArgs a, const __grid_constant_
           }
           const float m_tile = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3)) * scale2;     // -inf when the row sees nothing here
 
-          float m_cur = -INFINITY;
-          if (j > 0) {
-            ok = mbar_wait(&ctl->m_pub[wg ^ 1], n_other & 1, abort_flag);
-            if (!ok) break;
-            ++n_other;
-            m_cur = ctl->m_row[row_t];
-          }
           float m_new = m_cur;
           bool rescale = false;
           if (m_tile > m_cur + kRescaleThreshold || m_cur == -INFINITY) {
