@@ -37,7 +37,7 @@ WORKLOAD_DESC = ("c2: Llama-3.1-8B layer shape (32 q heads / 8 kv heads / dim 12
                  "draft KV 8x128 gather of 1024 tokens")
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel (attn_tc2_kernel), from the
 # ncu capture summarised in profiles/attn_tc2_kernel_c2_16k.md.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 69959424
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 69613056            # 67,914,496 read + 1,698,560 written
 NOMINAL = {"hbm_gbs": 7700.0, "tf": 2250.0}            # B200 data-sheet figures, for context only
 
 
